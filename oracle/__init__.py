@@ -1,0 +1,199 @@
+"""ctypes front end of the fp64 CPU oracle (``a2sf_oracle.c``).
+
+TEST INFRASTRUCTURE: only tests, the smoke check and the benchmark's CPU-baseline
+leg import this package.  It shares no code with the CUDA library and never
+imports it.  All arrays are numpy float64 / int32, C-contiguous.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "a2sf_oracle.c"
+_LIB_PATH = _HERE / "liba2sf_oracle.so"
+_lib = None
+
+_D = ctypes.POINTER(ctypes.c_double)
+_I = ctypes.POINTER(ctypes.c_int32)
+
+
+def build(force: bool = False, extra_cflags: Sequence[str] = (), out: Optional[Path] = None) -> Path:
+    """Compile the oracle with gcc (plain -O2, no fast-math: fp64 as written)."""
+    out = Path(out) if out else _LIB_PATH
+    if not force and out.exists() and out.stat().st_mtime >= _SRC.stat().st_mtime:
+        return out
+    tmp = out.with_suffix(f".tmp{os.getpid()}.so")
+    cmd = ["gcc", "-O2", "-fPIC", "-shared", "-std=c11", "-pthread", *extra_cflags,
+           str(_SRC), "-o", str(tmp), "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, out)
+    return out
+
+
+def _bind(lib):
+    c_int, c_dbl = ctypes.c_int, ctypes.c_double
+    lib.a2sf_oracle_softmax_row.restype = c_dbl
+    lib.a2sf_oracle_softmax_row.argtypes = [_D, _D, c_int, c_dbl, c_int, _D]
+    lib.a2sf_oracle_prefill_rows.restype = None
+    lib.a2sf_oracle_prefill_rows.argtypes = [_D, _D, _D, c_int, c_int, c_dbl, _D, c_int,
+                                             c_int, c_int, _D, _D, _D]
+    lib.a2sf_oracle_select.restype = c_int
+    lib.a2sf_oracle_select.argtypes = [_D, c_int, c_int, c_int, _I]
+    lib.a2sf_oracle_cache_load.restype = None
+    lib.a2sf_oracle_cache_load.argtypes = [_D, _D, _D, _I, c_int, c_int, c_int,
+                                           _D, _D, _D, _I, _I, _I]
+    lib.a2sf_oracle_decode_step.restype = None
+    lib.a2sf_oracle_decode_step.argtypes = [_D, _D, _D, _I, _I, _I, _D, _D, _D,
+                                            c_int, c_dbl, c_dbl, c_int, c_int, c_int,
+                                            _D, _I, _D]
+    lib.a2sf_oracle_prefill_batch.restype = c_int
+    lib.a2sf_oracle_prefill_batch.argtypes = [_D, _D, _D, c_int, c_int, c_int, c_dbl,
+                                              _D, c_int, c_int, c_int, c_int,
+                                              _D, _D, _D, _I, _I, c_int]
+    lib.a2sf_oracle_decode_step_batch.restype = c_int
+    lib.a2sf_oracle_decode_step_batch.argtypes = [_D, _D, _D, _I, _I, _I, _D, _D, _D,
+                                                  c_int, c_int, c_dbl, c_dbl, c_int, c_int,
+                                                  _I, _D, _I, _D, c_int]
+    return lib
+
+
+def load(path: Optional[Path] = None):
+    """Load (building if needed) the oracle library."""
+    global _lib
+    if path is not None:
+        return _bind(ctypes.CDLL(str(path)))
+    if _lib is None:
+        _lib = _bind(ctypes.CDLL(str(build())))
+    return _lib
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _dp(a: Optional[np.ndarray]):
+    return a.ctypes.data_as(_D) if a is not None else None
+
+
+def _ip(a: Optional[np.ndarray]):
+    return a.ctypes.data_as(_I) if a is not None else None
+
+
+def host_threads() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:  # pragma: no cover
+        return max(1, os.cpu_count() or 1)
+
+
+def attention_probs(Q, K, scale: float, lib=None) -> np.ndarray:
+    """Materialised causal softmax matrix P [n, n] (tiny inputs only)."""
+    lib = lib or load()
+    Q, K = _f64(Q), _f64(K)
+    n, d = Q.shape
+    P = np.zeros((n, n), dtype=np.float64)
+    for i in range(n):
+        lib.a2sf_oracle_softmax_row(_dp(Q), _dp(K), d, float(scale), i, _dp(P[i]))
+    return P
+
+
+def prefill_rows(Q, K, V, scale: float, alphas: Sequence[float], i0: int, i1: int, lib=None):
+    """Rows [i0, i1) of one unit: out rows, lse rows and their contribution to S."""
+    lib = lib or load()
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    n, d = Q.shape
+    al = _f64(list(alphas))
+    out = np.empty((i1 - i0, d), dtype=np.float64)
+    lse = np.empty((i1 - i0,), dtype=np.float64)
+    S = np.empty((len(al), n), dtype=np.float64)
+    lib.a2sf_oracle_prefill_rows(_dp(Q), _dp(K), _dp(V), n, d, float(scale), _dp(al), len(al),
+                                 int(i0), int(i1), _dp(out), _dp(lse), _dp(S))
+    return out, lse, S
+
+
+def select(S, M: int, R: int, lib=None) -> np.ndarray:
+    lib = lib or load()
+    S = _f64(S)
+    n = S.shape[0]
+    kept = np.empty((min(n, M),), dtype=np.int32)
+    m = lib.a2sf_oracle_select(_dp(S), n, int(M), int(R), _ip(kept))
+    assert m == kept.shape[0]
+    return kept
+
+
+def prefill(Q, K, V, scale: float, alphas: Sequence[float], M: int, R: int,
+            sel_alpha: int = 0, nthreads: int = 1, want_out: bool = True, lib=None):
+    """Full prefill of U units.  Q, K, V: [U, n, d].  Returns a dict with
+    out [U,n,d], lse [U,n], S [U,A,n], kept [U,min(n,M)] and the thread count used."""
+    lib = lib or load()
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    U, n, d = Q.shape
+    al = _f64(list(alphas))
+    A = len(al)
+    out = np.empty((U, n, d), dtype=np.float64) if want_out else None
+    lse = np.empty((U, n), dtype=np.float64)
+    S = np.empty((U, A, n), dtype=np.float64)
+    m = min(n, M)
+    kept = np.empty((U, m), dtype=np.int32)
+    kept_len = np.empty((U,), dtype=np.int32)
+    used = lib.a2sf_oracle_prefill_batch(_dp(Q), _dp(K), _dp(V), U, n, d, float(scale),
+                                         _dp(al), A, int(M), int(R), int(sel_alpha),
+                                         _dp(out), _dp(lse), _dp(S), _ip(kept), _ip(kept_len),
+                                         int(nthreads))
+    assert (kept_len == m).all()
+    return {"out": out, "lse": lse, "S": S, "kept": kept, "threads": used}
+
+
+class Cache:
+    """Slot-indexed pruned cache of U units, stepped by the oracle."""
+
+    def __init__(self, U: int, d: int, M: int, R: int, scale: float, lib=None):
+        self.lib = lib or load()
+        self.U, self.d, self.M, self.R, self.scale = U, d, M, R, float(scale)
+        self.K = np.zeros((U, M, d), dtype=np.float64)
+        self.V = np.zeros((U, M, d), dtype=np.float64)
+        self.S = np.zeros((U, M), dtype=np.float64)
+        self.pos = np.full((U, M), -1, dtype=np.int32)
+        self.count = np.zeros((U,), dtype=np.int32)
+        self.len = np.zeros((U,), dtype=np.int32)
+
+    def load(self, K, V, S, kept):
+        """K, V [U,n,d]; S [U,n]; kept [U,m]: slot s <- token kept[s]."""
+        K, V, S = _f64(K), _f64(V), _f64(S)
+        kept = np.ascontiguousarray(kept, dtype=np.int32)
+        U, n, d = K.shape
+        m = kept.shape[1]
+        for u in range(U):
+            self.lib.a2sf_oracle_cache_load(_dp(K[u]), _dp(V[u]), _dp(S[u]), _ip(kept[u]),
+                                            m, n, d, _dp(self.K[u]), _dp(self.V[u]),
+                                            _dp(self.S[u]), _ip(self.pos[u]),
+                                            _ip(self.count[u:u + 1]), _ip(self.len[u:u + 1]))
+
+    def step(self, q, k_new, v_new, alpha: float, force=None, nthreads: int = 1):
+        """One generation step for all units.  q, k_new, v_new: [U, d].
+        ``force`` [U] int32: slot to vacate instead of the rule's choice when the
+        cache is full (-3 = follow the rule).  Returns out [U,d], info [U,3]
+        (vacated, rule's choice, rule's runner-up) and their scores [U,3]."""
+        q, k_new, v_new = _f64(q), _f64(k_new), _f64(v_new)
+        out = np.empty((self.U, self.d), dtype=np.float64)
+        info = np.empty((self.U, 3), dtype=np.int32)
+        sc2 = np.empty((self.U, 3), dtype=np.float64)
+        f = None if force is None else np.ascontiguousarray(force, dtype=np.int32)
+        self.lib.a2sf_oracle_decode_step_batch(
+            _dp(self.K), _dp(self.V), _dp(self.S), _ip(self.pos), _ip(self.count), _ip(self.len),
+            _dp(q), _dp(k_new), _dp(v_new), self.U, self.d, self.scale, float(alpha),
+            self.M, self.R, _ip(f), _dp(out), _ip(info), _dp(sc2), int(nthreads))
+        return out, info, sc2
+
+    def snapshot(self):
+        return {k: getattr(self, k).copy() for k in ("K", "V", "S", "pos", "count", "len")}
+
+    def restore(self, snap):
+        for k, v in snap.items():
+            getattr(self, k)[...] = v
