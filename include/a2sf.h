@@ -1,0 +1,199 @@
+/*
+ * liba2sf -- C ABI of the A2SF KV-cache pruning hot path on one NVIDIA B200 (sm_100a).
+ *
+ * A2SF (Accumulative Attention Score with Forgetting Factor) keeps, per attention
+ * head, a score for every cached token: the forgetting-weighted sum over query
+ * steps of the softmax probability that token received (paper Eq. 5), and evicts
+ * the lowest-scoring tokens so the cache never exceeds a fixed budget (Sec. 3.1,
+ * Sec. 4.1).  This library computes, per (batch, head) unit:
+ *
+ *   prefill : causal attention over the prompt, the score of every prompt token,
+ *             and the set of tokens that stay in the cache;
+ *   decode  : one generation step over the pruned, slot-indexed cache -- attention,
+ *             the score recurrence S <- alpha*S + a_t, the eviction of one token
+ *             and the in-place insertion of the new one.
+ *
+ * Conventions
+ *   - Positions, slots and rows are 0-based.  n = prompt length, d = head size,
+ *     M = budget (cache slots per head), R = recent (newest positions that are
+ *     never evicted), U = B*H units.
+ *   - Unless an argument says "host", every data pointer is a DEVICE pointer owned
+ *     by the caller; the library never frees caller memory.  Rows of q/k/v/out
+ *     must be 16-byte aligned (base pointer and strides).
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and return without synchronising, except where stated.
+ *     The cache's resident count and length live on the device, so a decode step
+ *     has no host-side data-dependent control flow.
+ *   - Every function returns an a2sf_status.  Invalid arguments are rejected on
+ *     the host before anything is launched; nothing is dereferenced on the host.
+ *   - There is no CPU fallback.
+ */
+#ifndef A2SF_H
+#define A2SF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { A2SF_F32 = 0, A2SF_BF16 = 1, A2SF_F16 = 2 } a2sf_dtype;
+
+typedef enum {
+    A2SF_OK = 0,
+    A2SF_ERR_INVALID_ARG = -1,   /* null / misaligned pointer, bad shape or policy        */
+    A2SF_ERR_UNSUPPORTED = -2,   /* dtype or head size without a kernel                   */
+    A2SF_ERR_CUDA = -3,          /* a CUDA runtime call failed                            */
+    A2SF_ERR_TIMEOUT = -4,       /* a bounded device-side wait ran out (kernel gave up)   */
+    A2SF_ERR_WORKSPACE = -5      /* workspace / buffer smaller than the *_bytes() figure  */
+} a2sf_status;
+
+/* Shape and policy of a call.  `scale` = 0 selects 1/sqrt(d).  `alpha` is the
+ * forgetting factor of Eq. 5; the paper states 0 < alpha < 1 and also runs
+ * alpha = 0 (Sec. 4.4); alpha = 1 is the plain accumulative score of H2O (Eq. 4).
+ * Accepted: 0 <= alpha <= 1 with alpha^0 = 1.  budget >= 1, 0 <= recent <= budget,
+ * d in {64, 128}. */
+typedef struct a2sf_params {
+    int32_t B, H, d;
+    int32_t dtype;               /* a2sf_dtype of q, k, v, out and the cache rows */
+    int32_t budget, recent;
+    float alpha;
+    float scale;
+} a2sf_params;
+
+typedef struct a2sf_cache a2sf_cache;   /* opaque, owned by the library */
+
+/* ---------------------------------------------------------------------------
+ * Prefill (prompt phase).
+ *
+ * For every unit, with s_ij = scale * q_i . k_j for j <= i (causal mask: Eq. 3 sets
+ * the probability of a later key to zero) and P = row softmax of s:
+ *     out_i    = sum_j P_ij v_j
+ *     lse_i    = log sum_{j<=i} exp(s_ij)
+ *     scores_j = sum_{i>=j} alpha^(n-1-i) P_ij           (Eq. 5, Eq. 6: the sum ends
+ *                                                         at the diagonal term)
+ *     kept_idx = every position >= n-R plus, of the others, all but the n-M lowest
+ *                under the order (score, position) ascending; ascending positions.
+ *                If n <= M every position is kept.  (Sec. 3.1, Sec. 4.1)
+ *
+ * q, k, v, out : [B][H][n][d] in `dtype`, element strides stride_b/stride_h/stride_t,
+ *                d contiguous; out uses the same strides.
+ * scores       : [B][H][n] fp32, contiguous.      kept_idx: [B][H][min(n,M)] int32.
+ * lse_opt      : [B][H][n] fp32 or NULL (then it lives in the workspace).
+ * workspace    : device scratch of at least a2sf_prefill_workspace_bytes() bytes,
+ *                256-byte aligned; contents undefined afterwards.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA (launch failure).
+ * ------------------------------------------------------------------------- */
+size_t a2sf_prefill_workspace_bytes(const a2sf_params *p, int32_t n);
+
+int a2sf_prefill(const a2sf_params *p, int32_t n,
+                 const void *q, const void *k, const void *v,
+                 int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                 void *out, float *scores, int32_t *kept_idx, float *lse_opt,
+                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Scores and kept set only, from the log-sum-exp a prefill produced (the second
+ * pass of the prefill alone).  Lets a sweep over alpha reuse one attention pass.
+ * lse: [B][H][n] fp32 (input).  Other arguments as in a2sf_prefill; workspace may
+ * be NULL when a2sf_rescore_workspace_bytes() is 0. */
+size_t a2sf_rescore_workspace_bytes(const a2sf_params *p, int32_t n);
+
+int a2sf_rescore(const a2sf_params *p, int32_t n,
+                 const void *q, const void *k,
+                 int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                 const float *lse, float *scores, int32_t *kept_idx,
+                 void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Same as a2sf_prefill with HOST buffers: q, k, v, out contiguous [B][H][n][d];
+ * scores, kept_idx as above, all in host memory (pinned memory makes the copies
+ * asynchronous).  Inputs are copied to the device workspace, results copied back,
+ * and the call returns after the stream has drained.  The device copies of k, v,
+ * scores and kept_idx stay valid in the workspace for a2sf_cache_load: their
+ * addresses are returned through dev_k, dev_v, dev_scores, dev_kept (any may be NULL). */
+size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n);
+
+int a2sf_prefill_host(const a2sf_params *p, int32_t n,
+                      const void *q_host, const void *k_host, const void *v_host,
+                      void *out_host, float *scores_host, int32_t *kept_idx_host,
+                      void *workspace, size_t workspace_bytes,
+                      void **dev_k, void **dev_v, float **dev_scores, int32_t **dev_kept,
+                      void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * The pruned cache.  Per unit: K and V rows [M][d] in `dtype`, scores [M] fp32,
+ * positions [M] int32 (slot -> token position, -1 = empty), the resident count and
+ * the number of tokens seen so far.  Slot order carries no meaning (softmax . V is
+ * permutation invariant); positions exist for recency and the tie-break.
+ *
+ * a2sf_cache_create: `device_mem` NULL -> the library allocates a2sf_cache_bytes()
+ * with cudaMalloc and frees it in a2sf_cache_destroy; otherwise it adopts the
+ * caller's buffer (256-byte aligned, at least a2sf_cache_bytes(); WORKSPACE if
+ * smaller), which the caller frees after destroy.  The cache starts empty.
+ * Creation synchronises the device (it is not on the hot path).
+ * ------------------------------------------------------------------------- */
+size_t a2sf_cache_bytes(const a2sf_params *p);
+
+int a2sf_cache_create(const a2sf_params *p, void *device_mem, size_t bytes, a2sf_cache **cache);
+
+int a2sf_cache_destroy(a2sf_cache *cache);
+
+/* Initial cache from a prefill: slot s <- token kept_idx[s] (its K and V row, score
+ * and position); count = min(n, M); length = n; remaining slots emptied.
+ * k, v: [B][H][n][d] with the given strides; scores [B][H][n]; kept_idx [B][H][min(n,M)]. */
+int a2sf_cache_load(a2sf_cache *cache, int32_t n, const void *k, const void *v,
+                    int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                    const float *scores, const int32_t *kept_idx, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * One generation step for every unit, fused in one kernel (Eq. 5 as a recurrence;
+ * Sec. 3.1 eviction; the softmax runs over the pruned cache plus the new token,
+ * cf. Sec. 2.2 on the changed denominator):
+ *   a      = softmax over { scale*q.K[slot] : slot < count } and scale*q.k_new
+ *   out    = sum_slot a_slot V[slot] + a_self v_new
+ *   S[slot] <- alpha*S[slot] + a_slot,   S_new = a_self
+ *   count < M : the new token goes to slot `count`; evicted_slot = -1.
+ *   count = M : among the slots whose position is <= p - R (p = position of the new
+ *               token) -- and the new token itself iff R = 0 -- the minimum under
+ *               (S, position) is vacated and the new K/V/score/position are written
+ *               there in place; evicted_slot = that slot, or -2 if the new token was
+ *               the minimum (cache left as it was, apart from the updated scores).
+ *   length += 1.
+ * q, k_new, v_new, out: [B][H][d] contiguous in the cache's dtype; evicted_slot
+ * [B][H] int32.  alpha overrides the value given at creation.
+ * Steps on one cache must be ordered (same stream, or events between streams).
+ * ------------------------------------------------------------------------- */
+int a2sf_decode_step(a2sf_cache *cache, float alpha,
+                     const void *q, const void *k_new, const void *v_new,
+                     void *out, int32_t *evicted_slot, void *cuda_stream);
+
+/* The same step with HOST buffers (pinned for asynchronous copies): q, k_new, v_new
+ * are copied into staging rows inside the cache, the step runs, out and
+ * evicted_slot are copied back.  Returns after the stream has drained. */
+int a2sf_decode_step_host(a2sf_cache *cache, float alpha,
+                          const void *q_host, const void *k_new_host, const void *v_new_host,
+                          void *out_host, int32_t *evicted_slot_host, void *cuda_stream);
+
+/* Snapshot / restore of the whole cache state into / from caller DEVICE buffers:
+ * k, v [B][H][M][d] dtype; scores [B][H][M] fp32; pos [B][H][M] int32; count, len
+ * [B][H] int32.  Any pointer may be NULL to skip that part. */
+int a2sf_cache_export(const a2sf_cache *cache, void *k, void *v, float *scores,
+                      int32_t *pos, int32_t *count, int32_t *len, void *cuda_stream);
+
+int a2sf_cache_import(a2sf_cache *cache, const void *k, const void *v, const float *scores,
+                      const int32_t *pos, const int32_t *count, const int32_t *len,
+                      void *cuda_stream);
+
+/* Number of kernels this library has launched in the calling process so far. */
+int64_t a2sf_kernel_launch_count(void);
+
+/* Synchronises the stream and returns the sticky device-side status (A2SF_OK, or
+ * A2SF_ERR_TIMEOUT if a kernel abandoned a bounded wait), then clears it. */
+int a2sf_last_device_status(void *cuda_stream);
+
+const char *a2sf_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* A2SF_H */

@@ -1,0 +1,384 @@
+// Host side of the C ABI declared in include/a2sf.h: argument validation, the cache
+// object, workspace carving and kernel dispatch.  No data is touched on the host.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace a2sf {
+
+static std::atomic<int64_t> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+static inline int elem_bytes(int dtype) { return dtype == A2SF_F32 ? 4 : 2; }
+
+static int check_params(const a2sf_params *p)
+{
+    if (!p) return A2SF_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->budget < 1 || p->recent < 0 || p->recent > p->budget)
+        return A2SF_ERR_INVALID_ARG;
+    if (!(p->alpha >= 0.f && p->alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;   // rejects NaN
+    if (!(p->scale >= 0.f) || std::isinf(p->scale)) return A2SF_ERR_INVALID_ARG;
+    if (p->dtype != A2SF_F32 && p->dtype != A2SF_BF16 && p->dtype != A2SF_F16)
+        return A2SF_ERR_UNSUPPORTED;
+    if (p->d != 64 && p->d != 128) return A2SF_ERR_UNSUPPORTED;
+    if ((int64_t)p->B * p->H > 0x7fffffff) return A2SF_ERR_INVALID_ARG;
+    return A2SF_OK;
+}
+
+static inline float eff_scale(const a2sf_params *p)
+{
+    return p->scale > 0.f ? p->scale : 1.0f / std::sqrt((float)p->d);
+}
+
+static int check_strides(const a2sf_params *p, int64_t sb, int64_t sh, int64_t st)
+{
+    const int vec = 16 / elem_bytes(p->dtype);
+    if (st < p->d || sh < 1 || sb < 1) return A2SF_ERR_INVALID_ARG;
+    if (st % vec || sh % vec || sb % vec) return A2SF_ERR_INVALID_ARG;
+    return A2SF_OK;
+}
+
+// prefill workspace: the log-sum-exp rows when the caller does not keep them
+static size_t prefill_ws_bytes(const a2sf_params *p, int n)
+{
+    return align_up((size_t)p->B * p->H * n * sizeof(float));
+}
+
+static int run_scores_and_select(const a2sf_params *p, int n, PrefillArgs &a, int32_t *kept,
+                                 cudaStream_t s)
+{
+    if (launch_prefill_pass2_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    if (launch_select(a.scores, kept, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+}  // namespace a2sf
+
+using namespace a2sf;
+
+struct a2sf_cache {
+    a2sf_params p;
+    CacheView view;
+    void *mem;
+    size_t bytes;
+    bool owns;
+    // staging rows for the host-buffer step: q, k_new, v_new, out [U][d], evicted [U]
+    void *st_q, *st_k, *st_v, *st_out;
+    int32_t *st_ev;
+};
+
+extern "C" {
+
+size_t a2sf_prefill_workspace_bytes(const a2sf_params *p, int32_t n)
+{
+    if (check_params(p) != A2SF_OK || n < 1) return 0;
+    return prefill_ws_bytes(p, n);
+}
+
+size_t a2sf_rescore_workspace_bytes(const a2sf_params *p, int32_t n)
+{
+    (void)p; (void)n;
+    return 0;
+}
+
+int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
+                 int64_t stride_b, int64_t stride_h, int64_t stride_t, void *out, float *scores,
+                 int32_t *kept_idx, float *lse_opt, void *workspace, size_t workspace_bytes,
+                 void *cuda_stream)
+{
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    if ((rc = check_strides(p, stride_b, stride_h, stride_t)) != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) ||
+        !aligned(scores, 4) || !aligned(kept_idx, 4))
+        return A2SF_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256)) return A2SF_ERR_INVALID_ARG;
+    if (workspace_bytes < prefill_ws_bytes(p, n)) return A2SF_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+
+    PrefillArgs a;
+    a.q = q; a.k = k; a.v = v; a.out = out;
+    a.lse = lse_opt ? lse_opt : static_cast<float *>(workspace);
+    a.scores = scores;
+    a.st = Strides{stride_b, stride_h, stride_t};
+    a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
+    a.scale = eff_scale(p); a.alpha = p->alpha;
+    if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    return run_scores_and_select(p, n, a, kept_idx, s);
+}
+
+int a2sf_rescore(const a2sf_params *p, int32_t n, const void *q, const void *k, int64_t stride_b,
+                 int64_t stride_h, int64_t stride_t, const float *lse, float *scores,
+                 int32_t *kept_idx, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    (void)workspace; (void)workspace_bytes;
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (n < 1 || !q || !k || !lse || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    if ((rc = check_strides(p, stride_b, stride_h, stride_t)) != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16)) return A2SF_ERR_INVALID_ARG;
+    PrefillArgs a;
+    a.q = q; a.k = k; a.v = nullptr; a.out = nullptr;
+    a.lse = const_cast<float *>(lse);
+    a.scores = scores;
+    a.st = Strides{stride_b, stride_h, stride_t};
+    a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
+    a.scale = eff_scale(p); a.alpha = p->alpha;
+    return run_scores_and_select(p, n, a, kept_idx, static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n)
+{
+    if (check_params(p) != A2SF_OK || n < 1) return 0;
+    const size_t U = (size_t)p->B * p->H;
+    const size_t tensor = align_up(U * n * p->d * elem_bytes(p->dtype));
+    const size_t m = (size_t)(n < p->budget ? n : p->budget);
+    return 4 * tensor + align_up(U * n * 4) + align_up(U * m * 4) + prefill_ws_bytes(p, n);
+}
+
+int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const void *k_host,
+                      const void *v_host, void *out_host, float *scores_host,
+                      int32_t *kept_idx_host, void *workspace, size_t workspace_bytes,
+                      void **dev_k, void **dev_v, float **dev_scores, int32_t **dev_kept,
+                      void *cuda_stream)
+{
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (n < 1 || !q_host || !k_host || !v_host || !out_host || !scores_host || !kept_idx_host)
+        return A2SF_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256)) return A2SF_ERR_INVALID_ARG;
+    if (workspace_bytes < a2sf_prefill_host_workspace_bytes(p, n)) return A2SF_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t U = (size_t)p->B * p->H;
+    const size_t tbytes = U * n * p->d * elem_bytes(p->dtype);
+    const size_t tensor = align_up(tbytes);
+    const size_t m = (size_t)(n < p->budget ? n : p->budget);
+    char *base = static_cast<char *>(workspace);
+    void *dq = base, *dk = base + tensor, *dv = base + 2 * tensor, *dout = base + 3 * tensor;
+    float *dsc = reinterpret_cast<float *>(base + 4 * tensor);
+    int32_t *dkept = reinterpret_cast<int32_t *>(base + 4 * tensor + align_up(U * n * 4));
+    void *inner = base + 4 * tensor + align_up(U * n * 4) + align_up(U * m * 4);
+
+    if (cudaMemcpyAsync(dq, q_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dk, k_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    const int64_t st = p->d, sh = (int64_t)n * p->d, sb = (int64_t)p->H * n * p->d;
+    rc = a2sf_prefill(p, n, dq, dk, dv, sb, sh, st, dout, dsc, dkept, nullptr, inner,
+                      prefill_ws_bytes(p, n), cuda_stream);
+    if (rc != A2SF_OK) return rc;
+    if (cudaMemcpyAsync(out_host, dout, tbytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(scores_host, dsc, U * n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(kept_idx_host, dkept, U * m * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return A2SF_ERR_CUDA;
+    if (dev_k) *dev_k = dk;
+    if (dev_v) *dev_v = dv;
+    if (dev_scores) *dev_scores = dsc;
+    if (dev_kept) *dev_kept = dkept;
+    return A2SF_OK;
+}
+
+// ---- cache object --------------------------------------------------------------
+
+struct CacheLayout {
+    size_t K, V, S, pos, count, len, st_q, st_k, st_v, st_out, st_ev, total;
+};
+
+static CacheLayout cache_layout(const a2sf_params *p)
+{
+    const size_t U = (size_t)p->B * p->H, M = p->budget, d = p->d, e = elem_bytes(p->dtype);
+    CacheLayout L;
+    size_t off = 0;
+    L.K = off; off += align_up(U * M * d * e);
+    L.V = off; off += align_up(U * M * d * e);
+    L.S = off; off += align_up(U * M * 4);
+    L.pos = off; off += align_up(U * M * 4);
+    L.count = off; off += align_up(U * 4);
+    L.len = off; off += align_up(U * 4);
+    L.st_q = off; off += align_up(U * d * e);
+    L.st_k = off; off += align_up(U * d * e);
+    L.st_v = off; off += align_up(U * d * e);
+    L.st_out = off; off += align_up(U * d * e);
+    L.st_ev = off; off += align_up(U * 4);
+    L.total = off;
+    return L;
+}
+
+size_t a2sf_cache_bytes(const a2sf_params *p)
+{
+    if (check_params(p) != A2SF_OK) return 0;
+    return cache_layout(p).total;
+}
+
+int a2sf_cache_create(const a2sf_params *p, void *device_mem, size_t bytes, a2sf_cache **cache)
+{
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (!cache) return A2SF_ERR_INVALID_ARG;
+    *cache = nullptr;
+    const CacheLayout L = cache_layout(p);
+    a2sf_cache *c = new (std::nothrow) a2sf_cache;
+    if (!c) return A2SF_ERR_CUDA;
+    c->p = *p;
+    c->owns = device_mem == nullptr;
+    if (device_mem) {
+        if (!aligned(device_mem, 256)) { delete c; return A2SF_ERR_INVALID_ARG; }
+        if (bytes < L.total) { delete c; return A2SF_ERR_WORKSPACE; }
+        c->mem = device_mem;
+    } else if (cudaMalloc(&c->mem, L.total) != cudaSuccess) {
+        delete c;
+        return A2SF_ERR_CUDA;
+    }
+    c->bytes = L.total;
+    char *b = static_cast<char *>(c->mem);
+    c->view.K = b + L.K; c->view.V = b + L.V;
+    c->view.S = reinterpret_cast<float *>(b + L.S);
+    c->view.pos = reinterpret_cast<int32_t *>(b + L.pos);
+    c->view.count = reinterpret_cast<int32_t *>(b + L.count);
+    c->view.len = reinterpret_cast<int32_t *>(b + L.len);
+    c->view.U = p->B * p->H; c->view.M = p->budget; c->view.R = p->recent;
+    c->view.d = p->d; c->view.dtype = p->dtype; c->view.scale = eff_scale(p);
+    c->st_q = b + L.st_q; c->st_k = b + L.st_k; c->st_v = b + L.st_v; c->st_out = b + L.st_out;
+    c->st_ev = reinterpret_cast<int32_t *>(b + L.st_ev);
+    // empty cache: zero scores and counters, positions -1
+    if (cudaMemset(b + L.S, 0, L.st_q - L.S) != cudaSuccess ||
+        cudaMemset(b + L.pos, 0xff, L.count - L.pos) != cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess) {
+        if (c->owns) cudaFree(c->mem);
+        delete c;
+        return A2SF_ERR_CUDA;
+    }
+    *cache = c;
+    return A2SF_OK;
+}
+
+int a2sf_cache_destroy(a2sf_cache *cache)
+{
+    if (!cache) return A2SF_ERR_INVALID_ARG;
+    int rc = A2SF_OK;
+    if (cache->owns && cudaFree(cache->mem) != cudaSuccess) rc = A2SF_ERR_CUDA;
+    delete cache;
+    return rc;
+}
+
+int a2sf_cache_load(a2sf_cache *cache, int32_t n, const void *k, const void *v, int64_t stride_b,
+                    int64_t stride_h, int64_t stride_t, const float *scores,
+                    const int32_t *kept_idx, void *cuda_stream)
+{
+    if (!cache || n < 1 || !k || !v || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
+    if (rc != A2SF_OK) return rc;
+    if (!aligned(k, 16) || !aligned(v, 16)) return A2SF_ERR_INVALID_ARG;
+    if (launch_cache_load(cache->view, cache->p.H, n, k, v, Strides{stride_b, stride_h, stride_t},
+                          scores, kept_idx, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_decode_step(a2sf_cache *cache, float alpha, const void *q, const void *k_new,
+                     const void *v_new, void *out, int32_t *evicted_slot, void *cuda_stream)
+{
+    if (!cache || !q || !k_new || !v_new || !out || !evicted_slot) return A2SF_ERR_INVALID_ARG;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16))
+        return A2SF_ERR_INVALID_ARG;
+    if (launch_decode_step(cache->view, alpha, q, k_new, v_new, out, evicted_slot,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_decode_step_host(a2sf_cache *cache, float alpha, const void *q_host,
+                          const void *k_new_host, const void *v_new_host, void *out_host,
+                          int32_t *evicted_slot_host, void *cuda_stream)
+{
+    if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !evicted_slot_host)
+        return A2SF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t U = cache->view.U;
+    const size_t row = U * cache->p.d * elem_bytes(cache->p.dtype);
+    if (cudaMemcpyAsync(cache->st_q, q_host, row, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(cache->st_k, k_new_host, row, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(cache->st_v, v_new_host, row, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    int rc = a2sf_decode_step(cache, alpha, cache->st_q, cache->st_k, cache->st_v, cache->st_out,
+                              cache->st_ev, cuda_stream);
+    if (rc != A2SF_OK) return rc;
+    if (cudaMemcpyAsync(out_host, cache->st_out, row, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(evicted_slot_host, cache->st_ev, U * 4, cudaMemcpyDeviceToHost, s) !=
+            cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return cudaStreamSynchronize(s) == cudaSuccess ? A2SF_OK : A2SF_ERR_CUDA;
+}
+
+static int copy_part(void *dst, const void *src, size_t bytes, cudaStream_t s)
+{
+    if (!dst || !src) return A2SF_OK;
+    return cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, s) == cudaSuccess
+               ? A2SF_OK : A2SF_ERR_CUDA;
+}
+
+int a2sf_cache_export(const a2sf_cache *cache, void *k, void *v, float *scores, int32_t *pos,
+                      int32_t *count, int32_t *len, void *cuda_stream)
+{
+    if (!cache) return A2SF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const CacheView &c = cache->view;
+    const size_t U = c.U, M = c.M, rows = U * M * c.d * elem_bytes(c.dtype);
+    int rc = copy_part(k, c.K, rows, s);
+    if (rc == A2SF_OK) rc = copy_part(v, c.V, rows, s);
+    if (rc == A2SF_OK) rc = copy_part(scores, c.S, U * M * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(pos, c.pos, U * M * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(count, c.count, U * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(len, c.len, U * 4, s);
+    return rc;
+}
+
+int a2sf_cache_import(a2sf_cache *cache, const void *k, const void *v, const float *scores,
+                      const int32_t *pos, const int32_t *count, const int32_t *len,
+                      void *cuda_stream)
+{
+    if (!cache) return A2SF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const CacheView &c = cache->view;
+    const size_t U = c.U, M = c.M, rows = U * M * c.d * elem_bytes(c.dtype);
+    int rc = copy_part(c.K, k, rows, s);
+    if (rc == A2SF_OK) rc = copy_part(c.V, v, rows, s);
+    if (rc == A2SF_OK) rc = copy_part(c.S, scores, U * M * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(c.pos, pos, U * M * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(c.count, count, U * 4, s);
+    if (rc == A2SF_OK) rc = copy_part(c.len, len, U * 4, s);
+    return rc;
+}
+
+int64_t a2sf_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int a2sf_last_device_status(void *cuda_stream)
+{
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+const char *a2sf_status_string(int status)
+{
+    switch (status) {
+    case A2SF_OK: return "ok";
+    case A2SF_ERR_INVALID_ARG: return "invalid argument";
+    case A2SF_ERR_UNSUPPORTED: return "unsupported dtype or head size";
+    case A2SF_ERR_CUDA: return "CUDA runtime error";
+    case A2SF_ERR_TIMEOUT: return "device-side wait timed out";
+    case A2SF_ERR_WORKSPACE: return "workspace too small";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,132 @@
+// Shared device/host helpers of liba2sf (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/a2sf.h"
+
+namespace a2sf {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Strided view of a [B][H][n][d] tensor; strides in elements, d contiguous.
+struct Strides {
+    int64_t b, h, t;
+};
+
+// ---- element traits: 16-byte vector <-> fp32 --------------------------------
+template <typename T> struct Elem;
+
+template <> struct Elem<float> {
+    static constexpr int kVec = 4;   // elements per 16 bytes
+    __device__ static void unpack(const uint4 &r, float *f)
+    {
+        f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+    }
+    __device__ static float to_float(float x) { return x; }
+    __device__ static float from_float(float x) { return x; }
+};
+
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kVec = 8;
+    __device__ static void unpack(const uint4 &r, float *f)
+    {
+        // a bf16 is the upper half of an fp32
+        f[0] = __uint_as_float(r.x << 16); f[1] = __uint_as_float(r.x & 0xffff0000u);
+        f[2] = __uint_as_float(r.y << 16); f[3] = __uint_as_float(r.y & 0xffff0000u);
+        f[4] = __uint_as_float(r.z << 16); f[5] = __uint_as_float(r.z & 0xffff0000u);
+        f[6] = __uint_as_float(r.w << 16); f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+    __device__ static float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+    __device__ static __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+};
+
+template <> struct Elem<__half> {
+    static constexpr int kVec = 8;
+    __device__ static void unpack(const uint4 &r, float *f)
+    {
+        const __half2 *h = reinterpret_cast<const __half2 *>(&r);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float2 t = __half22float2(h[i]);
+            f[2 * i] = t.x; f[2 * i + 1] = t.y;
+        }
+    }
+    __device__ static float to_float(__half x) { return __half2float(x); }
+    __device__ static __half from_float(float x) { return __float2half_rn(x); }
+};
+
+// streaming 16-byte load that does not displace L1 lines
+__device__ __forceinline__ uint4 ld_stream16(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        unsigned long long t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = t < v ? t : v;
+    }
+    return v;
+}
+
+// ---- host-side launch bookkeeping -------------------------------------------
+void count_launch(int n = 1);
+
+// ---- kernel launchers (one per translation unit) -----------------------------
+struct PrefillArgs {
+    const void *q, *k, *v;
+    void *out;
+    float *lse;        // [U][n]
+    float *scores;     // [U][n]
+    Strides st;
+    int B, H, n, d;
+    float scale, alpha;
+};
+
+cudaError_t launch_prefill_pass1_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
+cudaError_t launch_prefill_pass2_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
+
+cudaError_t launch_select(const float *scores, int32_t *kept, int U, int n, int M, int R,
+                          cudaStream_t s);
+
+struct CacheView {
+    void *K, *V;          // [U][M][d]
+    float *S;             // [U][M]
+    int32_t *pos;         // [U][M]
+    int32_t *count, *len; // [U]
+    int U, M, R, d, dtype;
+    float scale;
+};
+
+cudaError_t launch_cache_load(const CacheView &c, int H, int n, const void *k, const void *v,
+                              Strides st, const float *scores, const int32_t *kept,
+                              cudaStream_t s);
+
+cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
+                               const void *v_new, void *out, int32_t *evicted, cudaStream_t s);
+
+}  // namespace a2sf

@@ -1,0 +1,251 @@
+// Fused A2SF generation step (one kernel): attention over the pruned, slot-indexed
+// cache + the new token, score recurrence S <- alpha*S + a (paper Eq. 5 written as a
+// recurrence), argmin eviction under (S, position) over the non-recent slots
+// (Sec. 3.1, Sec. 4.1) and the in-place write of the new K/V row.
+//
+// Memory-bound: every K and V row of the head is read exactly once with 16-byte
+// loads, lanes laid across the row so a warp reads whole 512-byte spans.
+#include "common.cuh"
+
+namespace a2sf {
+
+namespace {
+
+constexpr int kDecodeThreads = 256;
+constexpr int kUnroll = 4;
+
+template <int NT>
+__device__ __forceinline__ float block_max(float v, float *red)
+{
+    v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = red[0];
+#pragma unroll
+    for (int w = 1; w < NT / 32; ++w) r = fmaxf(r, red[w]);
+    return r;
+}
+
+template <int NT>
+__device__ __forceinline__ float block_sum(float v, float *red)
+{
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = red[0];
+#pragma unroll
+    for (int w = 1; w < NT / 32; ++w) r += red[w];   // fixed order: run-to-run identical
+    return r;
+}
+
+template <typename T, int D, int NT>
+__global__ void __launch_bounds__(NT)
+decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *__restrict__ k_new,
+                   const T *__restrict__ v_new, T *__restrict__ out, int32_t *__restrict__ evicted)
+{
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int LPR = D / VEC;          // lanes per row
+    constexpr int RPW = 32 / LPR;         // rows per warp-wide load
+    constexpr int NW = NT / 32;
+    static_assert(LPR <= 32 && 32 % LPR == 0, "row must fit a warp");
+
+    extern __shared__ float smem[];
+    const int M = c.M;
+    float *w = smem;                       // [M+1] logits, then exp(logit - max)
+    float *part = w + ((M + 1 + 3) & ~3);  // [NW][D] partial outputs
+    float *red = part + NW * D;            // [NW] reduction scratch
+    __shared__ unsigned long long red_key[NW];
+    __shared__ int s_target;
+
+    const int u = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int cnt = c.count[u];
+    const int p = c.len[u];
+
+    T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
+    T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
+    float *Su = c.S + (size_t)u * M;
+    int32_t *posu = c.pos + (size_t)u * M;
+
+    float qf[VEC];
+    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
+
+    // ---- (i) logits against every resident key, and against the new key -------
+    const int ngroups = (cnt + RPW - 1) / RPW;
+    for (int g = warp; g < ngroups; g += NW * kUnroll) {
+        uint4 r[kUnroll];
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int row = (g + x * NW) * RPW + rsel;
+            r[x] = make_uint4(0, 0, 0, 0);
+            if (row < cnt) r[x] = ld_stream16(Ku + (size_t)row * D + sub * VEC);
+        }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int row = (g + x * NW) * RPW + rsel;
+            float kf[VEC];
+            Elem<T>::unpack(r[x], kf);
+            float dot = 0.f;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+            for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (sub == 0 && row < cnt) w[row] = dot * c.scale;
+        }
+    }
+    if (warp == 0) {
+        float kf[VEC];
+        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC), kf);
+        float dot = 0.f;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        if (lane == 0) w[cnt] = dot * c.scale;
+    }
+    __syncthreads();
+
+    // ---- (ii) softmax over resident + self ------------------------------------
+    float m = -INFINITY;
+    for (int s = tid; s <= cnt; s += NT) m = fmaxf(m, w[s]);
+    m = block_max<NT>(m, red);
+    float l = 0.f;
+    for (int s = tid; s <= cnt; s += NT) {
+        const float e = expf(w[s] - m);
+        w[s] = e;
+        l += e;
+    }
+    l = block_sum<NT>(l, red);
+    const float e_self = w[cnt];
+
+    // ---- (iii) out = (sum_s e_s V[s] + e_self v_new) / l ------------------------
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    for (int g = warp; g < ngroups; g += NW * kUnroll) {
+        uint4 r[kUnroll];
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int row = (g + x * NW) * RPW + rsel;
+            r[x] = make_uint4(0, 0, 0, 0);
+            if (row < cnt) r[x] = ld_stream16(Vu + (size_t)row * D + sub * VEC);
+        }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int row = (g + x * NW) * RPW + rsel;
+            const float ws = row < cnt ? w[row] : 0.f;
+            float vf[VEC];
+            Elem<T>::unpack(r[x], vf);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(ws, vf[e], acc[e]);
+        }
+    }
+#pragma unroll
+    for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+    if (rsel == 0)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) part[warp * D + sub * VEC + e] = acc[e];
+    __syncthreads();
+    if (tid < D) {
+        float o = 0.f;
+#pragma unroll
+        for (int x = 0; x < NW; ++x) o += part[x * D + tid];
+        o = fmaf(e_self, Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+        out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
+    }
+
+    // ---- (iv) S <- alpha*S + a ; (v) argmin over the non-recent slots ------------
+    const bool full = cnt >= M;
+    const int newest_evictable = p - c.R;     // candidates: position <= p - R
+    unsigned long long best = ~0ull;
+    int best_slot = -1;
+    for (int s = tid; s < cnt; s += NT) {
+        const float a = w[s] / l;
+        const float sn = fmaf(alpha, Su[s], a);
+        Su[s] = sn;
+        const int ps = posu[s];
+        if (full && ps <= newest_evictable) {
+            // scores are >= 0, so their bit patterns order like the values
+            const unsigned long long key =
+                ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
+            if (key < best) { best = key; best_slot = s; }
+        }
+    }
+    const float a_self = e_self / l;
+    const unsigned long long wbest = warp_min_u64(best);
+    if (lane == 0) red_key[warp] = wbest;
+    if (tid == 0) s_target = full ? -2 : cnt;
+    __syncthreads();
+    unsigned long long gbest = red_key[0];
+#pragma unroll
+    for (int x = 1; x < NW; ++x) gbest = red_key[x] < gbest ? red_key[x] : gbest;
+    if (full && best_slot >= 0 && best == gbest) {
+        // positions are distinct, so exactly one thread holds the minimum
+        const unsigned long long self_key =
+            ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
+        if (c.R > 0 || gbest < self_key) s_target = best_slot;
+    }
+    __syncthreads();
+
+    // ---- in-place insertion of the new token --------------------------------------
+    const int target = s_target;
+    if (target >= 0) {
+        if (tid < LPR)
+            *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
+                *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
+        else if (tid < 2 * LPR)
+            *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
+                *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
+    }
+    if (tid == 0) {
+        if (target >= 0) {
+            Su[target] = a_self;
+            posu[target] = p;
+        }
+        if (!full) c.count[u] = cnt + 1;
+        c.len[u] = p + 1;
+        evicted[u] = full ? target : -1;
+    }
+}
+
+template <typename T, int D>
+cudaError_t launch_typed(const CacheView &c, float alpha, const void *q, const void *k_new,
+                         const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    constexpr int NT = kDecodeThreads;
+    const size_t smem = (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 + (size_t)(NT / 32) * D * 4 +
+                        (NT / 32) * 4;
+    auto kern = decode_step_kernel<T, D, NT>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<c.U, NT, smem, s>>>(c, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
+                               static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
+                               const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+#define A2SF_DISPATCH(T)                                                                     \
+    (c.d == 64 ? launch_typed<T, 64>(c, alpha, q, k_new, v_new, out, evicted, s)             \
+               : launch_typed<T, 128>(c, alpha, q, k_new, v_new, out, evicted, s))
+    switch (c.dtype) {
+    case A2SF_F32: return A2SF_DISPATCH(float);
+    case A2SF_BF16: return A2SF_DISPATCH(__nv_bfloat16);
+    default: return A2SF_DISPATCH(__half);
+    }
+#undef A2SF_DISPATCH
+}
+
+}  // namespace a2sf
