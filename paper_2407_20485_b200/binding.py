@@ -1,0 +1,248 @@
+"""Thin ctypes binding over ``liba2sf.so`` (see ``include/a2sf.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch supplies device memory and streams.  There is no fallback: if the
+library has not been built this module raises on import.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+_LIB_PATH = Path(__file__).resolve().parent / "liba2sf.so"
+
+A2SF_F32, A2SF_BF16, A2SF_F16 = 0, 1, 2
+_DTYPE_CODE = {torch.float32: A2SF_F32, torch.bfloat16: A2SF_BF16, torch.float16: A2SF_F16}
+
+A2SF_OK = 0
+A2SF_ERR_INVALID_ARG, A2SF_ERR_UNSUPPORTED, A2SF_ERR_CUDA = -1, -2, -3
+A2SF_ERR_TIMEOUT, A2SF_ERR_WORKSPACE = -4, -5
+
+
+class a2sf_params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("budget", ctypes.c_int32), ("recent", ctypes.c_int32),
+                ("alpha", ctypes.c_float), ("scale", ctypes.c_float)]
+
+
+class A2SFError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def _load():
+    if not _LIB_PATH.exists():
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2407_20485_b200.build` "
+            "(there is no CPU fallback)")
+    lib = ctypes.CDLL(str(_LIB_PATH))
+    vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
+                             ctypes.c_size_t)
+    pp = ctypes.POINTER(a2sf_params)
+    pvp = ctypes.POINTER(vp)
+    sigs = {
+        "a2sf_prefill_workspace_bytes": (sz, [pp, i32]),
+        "a2sf_prefill": (ctypes.c_int, [pp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]),
+        "a2sf_rescore_workspace_bytes": (sz, [pp, i32]),
+        "a2sf_rescore": (ctypes.c_int, [pp, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]),
+        "a2sf_prefill_host_workspace_bytes": (sz, [pp, i32]),
+        "a2sf_prefill_host": (ctypes.c_int, [pp, i32, vp, vp, vp, vp, vp, vp, vp, sz,
+                                             pvp, pvp, pvp, pvp, vp]),
+        "a2sf_cache_bytes": (sz, [pp]),
+        "a2sf_cache_create": (ctypes.c_int, [pp, vp, sz, pvp]),
+        "a2sf_cache_destroy": (ctypes.c_int, [vp]),
+        "a2sf_cache_load": (ctypes.c_int, [vp, i32, vp, vp, i64, i64, i64, vp, vp, vp]),
+        "a2sf_decode_step": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
+        "a2sf_decode_step_host": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
+        "a2sf_cache_export": (ctypes.c_int, [vp] * 8),
+        "a2sf_cache_import": (ctypes.c_int, [vp] * 8),
+        "a2sf_kernel_launch_count": (ctypes.c_int64, []),
+        "a2sf_last_device_status": (ctypes.c_int, [vp]),
+        "a2sf_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(lib, name)
+        fn.restype, fn.argtypes = res, args
+    return lib, tuple(sigs)
+
+
+lib, EXPORTED = _load()
+
+
+def status_string(status: int) -> str:
+    return lib.a2sf_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != A2SF_OK:
+        raise A2SFError(status, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return ctypes.c_void_p(t)
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def make_params(B: int, H: int, d: int, dtype: torch.dtype, budget: int, recent: int,
+                alpha: float, scale: float = 0.0) -> a2sf_params:
+    return a2sf_params(B, H, d, _DTYPE_CODE[dtype], budget, recent, alpha, scale)
+
+
+def a2sf_kernel_launch_count() -> int:
+    return int(lib.a2sf_kernel_launch_count())
+
+
+def a2sf_last_device_status(stream=None) -> int:
+    return int(lib.a2sf_last_device_status(_stream(stream)))
+
+
+def a2sf_prefill_workspace_bytes(p: a2sf_params, n: int) -> int:
+    return int(lib.a2sf_prefill_workspace_bytes(ctypes.byref(p), n))
+
+
+def a2sf_rescore_workspace_bytes(p: a2sf_params, n: int) -> int:
+    return int(lib.a2sf_rescore_workspace_bytes(ctypes.byref(p), n))
+
+
+def _strides(t: torch.Tensor):
+    assert t.dim() == 4 and t.stride(3) == 1, "expected [B,H,n,d] with contiguous d"
+    return t.stride(0), t.stride(1), t.stride(2)
+
+
+def a2sf_prefill(p: a2sf_params, q, k, v, out=None, scores=None, kept_idx=None, lse=None,
+                 workspace=None, stream=None):
+    """q, k, v: device [B,H,n,d].  Returns (out, scores, kept_idx, lse)."""
+    B, H, n, d = q.shape
+    assert k.shape == q.shape and v.shape == q.shape
+    assert _strides(k) == _strides(q) and _strides(v) == _strides(q)
+    dev = q.device
+    m = min(n, p.budget)
+    out = torch.empty_like(q) if out is None else out
+    assert _strides(out) == _strides(q)
+    scores = torch.empty((B, H, n), dtype=torch.float32, device=dev) if scores is None else scores
+    kept_idx = torch.empty((B, H, m), dtype=torch.int32, device=dev) if kept_idx is None else kept_idx
+    lse = torch.empty((B, H, n), dtype=torch.float32, device=dev) if lse is None else lse
+    if workspace is None:
+        need = a2sf_prefill_workspace_bytes(p, n)
+        workspace = torch.empty((max(need, 256),), dtype=torch.uint8, device=dev)
+    sb, sh, st = _strides(q)
+    _check(lib.a2sf_prefill(ctypes.byref(p), n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st, _ptr(out),
+                            _ptr(scores), _ptr(kept_idx), _ptr(lse), _ptr(workspace),
+                            workspace.numel(), _stream(stream)), "a2sf_prefill")
+    return out, scores, kept_idx, lse
+
+
+def a2sf_rescore(p: a2sf_params, q, k, lse, scores=None, kept_idx=None, workspace=None,
+                 stream=None):
+    """Scores and kept set for ``p.alpha`` from an existing log-sum-exp."""
+    B, H, n, d = q.shape
+    dev = q.device
+    m = min(n, p.budget)
+    scores = torch.empty((B, H, n), dtype=torch.float32, device=dev) if scores is None else scores
+    kept_idx = torch.empty((B, H, m), dtype=torch.int32, device=dev) if kept_idx is None else kept_idx
+    sb, sh, st = _strides(q)
+    assert _strides(k) == (sb, sh, st)
+    if workspace is None:
+        need = a2sf_rescore_workspace_bytes(p, n)
+        workspace = torch.empty((need,), dtype=torch.uint8, device=dev) if need else None
+    _check(lib.a2sf_rescore(ctypes.byref(p), n, _ptr(q), _ptr(k), sb, sh, st, _ptr(lse),
+                            _ptr(scores), _ptr(kept_idx), _ptr(workspace),
+                            workspace.numel() if workspace is not None else 0,
+                            _stream(stream)), "a2sf_rescore")
+    return scores, kept_idx
+
+
+def a2sf_prefill_host_workspace_bytes(p: a2sf_params, n: int) -> int:
+    return int(lib.a2sf_prefill_host_workspace_bytes(ctypes.byref(p), n))
+
+
+def a2sf_prefill_host(p: a2sf_params, n: int, q_host, k_host, v_host, out_host, scores_host,
+                      kept_host, workspace, stream=None):
+    """Host-buffer prefill.  Returns the device addresses (ints) of k, v, scores,
+    kept_idx inside ``workspace`` for a following ``a2sf_cache_load``."""
+    dk, dv, ds, dkept = (ctypes.c_void_p() for _ in range(4))
+    _check(lib.a2sf_prefill_host(ctypes.byref(p), n, _ptr(q_host), _ptr(k_host), _ptr(v_host),
+                                 _ptr(out_host), _ptr(scores_host), _ptr(kept_host),
+                                 _ptr(workspace), workspace.numel(), ctypes.byref(dk),
+                                 ctypes.byref(dv), ctypes.byref(ds), ctypes.byref(dkept),
+                                 _stream(stream)), "a2sf_prefill_host")
+    return dk.value, dv.value, ds.value, dkept.value
+
+
+class Cache:
+    """Owner of an ``a2sf_cache`` whose storage is a torch device buffer."""
+
+    def __init__(self, p: a2sf_params, device="cuda"):
+        self.p = p
+        self.bytes = int(lib.a2sf_cache_bytes(ctypes.byref(p)))
+        if self.bytes == 0:
+            raise A2SFError(A2SF_ERR_INVALID_ARG, "a2sf_cache_bytes")
+        self.mem = torch.empty((self.bytes,), dtype=torch.uint8, device=device)
+        h = ctypes.c_void_p()
+        _check(lib.a2sf_cache_create(ctypes.byref(p), _ptr(self.mem), self.bytes, ctypes.byref(h)),
+               "a2sf_cache_create")
+        self.handle = h
+        self.U, self.M, self.d = p.B * p.H, p.budget, p.d
+        self.torch_dtype = {v: k for k, v in _DTYPE_CODE.items()}[p.dtype]
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.a2sf_cache_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    def a2sf_cache_load(self, k, v, scores, kept_idx, n=None, strides=None, stream=None):
+        """k, v: device tensors [B,H,n,d] (or raw addresses with ``n`` and ``strides``)."""
+        if isinstance(k, torch.Tensor):
+            n = k.shape[2]
+            strides = _strides(k)
+        sb, sh, st = strides
+        _check(lib.a2sf_cache_load(self.handle, n, _ptr(k), _ptr(v), sb, sh, st, _ptr(scores),
+                                   _ptr(kept_idx), _stream(stream)), "a2sf_cache_load")
+
+    def a2sf_decode_step(self, alpha, q, k_new, v_new, out, evicted, stream=None):
+        _check(lib.a2sf_decode_step(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                    _ptr(out), _ptr(evicted), _stream(stream)), "a2sf_decode_step")
+
+    def a2sf_decode_step_host(self, alpha, q, k_new, v_new, out, evicted, stream=None):
+        _check(lib.a2sf_decode_step_host(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                         _ptr(out), _ptr(evicted), _stream(stream)),
+               "a2sf_decode_step_host")
+
+    def state_tensors(self, device=None):
+        device = device or self.mem.device
+        B, H, M, d = self.p.B, self.p.H, self.M, self.d
+        return {
+            "k": torch.empty((B, H, M, d), dtype=self.torch_dtype, device=device),
+            "v": torch.empty((B, H, M, d), dtype=self.torch_dtype, device=device),
+            "scores": torch.empty((B, H, M), dtype=torch.float32, device=device),
+            "pos": torch.empty((B, H, M), dtype=torch.int32, device=device),
+            "count": torch.empty((B, H), dtype=torch.int32, device=device),
+            "len": torch.empty((B, H), dtype=torch.int32, device=device),
+        }
+
+    def a2sf_cache_export(self, state=None, stream=None):
+        state = state or self.state_tensors()
+        _check(lib.a2sf_cache_export(self.handle, *(_ptr(state.get(k)) for k in
+                                                    ("k", "v", "scores", "pos", "count", "len")),
+                                     _stream(stream)), "a2sf_cache_export")
+        return state
+
+    def a2sf_cache_import(self, state, stream=None):
+        _check(lib.a2sf_cache_import(self.handle, *(_ptr(state.get(k)) for k in
+                                                    ("k", "v", "scores", "pos", "count", "len")),
+                                     _stream(stream)), "a2sf_cache_import")
