@@ -130,7 +130,8 @@ def a2sf_prefill(p: a2sf_params, q, k, v, out=None, scores=None, kept_idx=None, 
     assert _strides(k) == _strides(q) and _strides(v) == _strides(q)
     dev = q.device
     m = min(n, p.budget)
-    out = torch.empty_like(q) if out is None else out
+    if out is None:
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=dev)
     assert _strides(out) == _strides(q)
     scores = torch.empty((B, H, n), dtype=torch.float32, device=dev) if scores is None else scores
     kept_idx = torch.empty((B, H, m), dtype=torch.int32, device=dev) if kept_idx is None else kept_idx

@@ -90,7 +90,6 @@ def test_strided_inputs_and_determinism():
     qs, ks, vs = view(q), view(k), view(v)
     p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
     o1, s1, k1, l1 = a2sf.a2sf_prefill(p, q, k, v)
-    o2 = torch.zeros_like(qs)
     o2 = view(torch.zeros_like(q))
     _, s2, k2, l2 = a2sf.a2sf_prefill(p, qs, ks, vs, out=o2)
     o3, s3, k3, l3 = a2sf.a2sf_prefill(p, q, k, v)
