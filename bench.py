@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the A2SF hot path: one "step" = prefill (attention + scores +
+selection) + cache build + T fused decode steps over one synthetic batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line.  `value` is the decode-step throughput in algorithmic GB/s
+(inputs resident in HBM); `prefill` carries the prefill-scoring TFLOP/s; `e2e` is
+the same decode metric through the host-buffer entry points (copies timed);
+`roofline` is the decode kernel against the measured HBM copy bandwidth;
+`cpu_baseline` is the fp64 oracle timed on the host cores on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import torch  # noqa: E402
+
+from paper_2407_20485_b200 import dist as a2dist  # noqa: E402
+from paper_2407_20485_b200 import workloads as wl  # noqa: E402
+
+METRIC = "a2sf_decode_step_hbm_gbps"
+UNIT = "GB/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+
+
+def load_peaks():
+    f = ROOT / "MEASURED_PEAKS.json"
+    if f.exists():
+        d = json.loads(f.read_text())
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.path or not os.path.exists(self.path):
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            # the region is busy throughout: the median describes the clocks under load
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def cuda_events(n):
+    return [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+
+
+def run_ours(args):
+    from paper_2407_20485_b200 import binding as a2sf   # raises if the CUDA library is missing
+
+    rank, local_rank, world = a2dist.init("nccl")
+    assert world == args.gpus, f"--gpus {args.gpus} but WORLD_SIZE={world}"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    w = wl.WORKLOADS[args.workload]
+    T = args.decode_steps or w.steps
+    # weak scaling: every rank owns a full per-GPU batch of a job world x as large
+    wg = w.scaled(B=w.B * world, steps=T)
+    b_range = a2dist.rank_batch_range(w.B, rank)
+    q, k, v = wl.make_prompt_chunked(wg, dev, b_range=b_range)
+    dq, dk, dv = wl.make_decode(wg, dev, t_range=(0, T), b_range=b_range)
+    U, n, d = w.units, w.n, w.d
+    p = a2sf.make_params(w.B, w.H, d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    m = min(n, w.budget)
+    out = torch.empty_like(q)
+    scores = torch.empty((w.B, w.H, n), dtype=torch.float32, device=dev)
+    kept = torch.empty((w.B, w.H, m), dtype=torch.int32, device=dev)
+    lse = torch.empty((w.B, w.H, n), dtype=torch.float32, device=dev)
+    ws = torch.empty((max(256, a2sf.a2sf_prefill_workspace_bytes(p, n)),), dtype=torch.uint8, device=dev)
+    cache = a2sf.Cache(p, dev)
+    o_t = torch.empty((T, w.B, w.H, d), dtype=w.torch_dtype, device=dev)
+    e_t = torch.empty((T, w.B, w.H), dtype=torch.int32, device=dev)
+
+    def step(ev=None):
+        if ev: ev[0].record()
+        a2sf.a2sf_prefill(p, q, k, v, out=out, scores=scores, kept_idx=kept, lse=lse, workspace=ws)
+        if ev: ev[1].record()
+        cache.a2sf_cache_load(k, v, scores, kept)
+        if ev: ev[2].record()
+        for t in range(T):
+            cache.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o_t[t], e_t[t])
+        if ev: ev[3].record()
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    a2dist.barrier()
+    evs = [cuda_events(4) for _ in range(args.steps)]
+    launches0 = a2sf.a2sf_kernel_launch_count()
+    with ClockSampler(local_rank) as clk:
+        torch.cuda.synchronize()
+        t_start = cuda_events(1)[0]
+        t_end = cuda_events(1)[0]
+        t_start.record()
+        for i in range(args.steps):
+            step(evs[i])
+        t_end.record()
+        torch.cuda.synchronize()
+    a2dist.barrier()
+    launches = a2sf.a2sf_kernel_launch_count() - launches0
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+    total_ms = t_start.elapsed_time(t_end)
+    prefill_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
+    load_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
+    decode_ms = sum(e[2].elapsed_time(e[3]) for e in evs)
+    clocks = clk.summary()
+
+    # ---- end to end through the host-buffer entry points (copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+        hout = torch.empty_like(hq).pin_memory()
+        hs = torch.empty((w.B, w.H, n), dtype=torch.float32).pin_memory()
+        hkept = torch.empty((w.B, w.H, m), dtype=torch.int32).pin_memory()
+        hdq, hdk, hdv = (t.cpu().pin_memory() for t in (dq, dk, dv))
+        ho = torch.empty((w.B, w.H, d), dtype=w.torch_dtype).pin_memory()
+        he = torch.empty((w.B, w.H), dtype=torch.int32).pin_memory()
+        del out
+        hws = torch.empty((a2sf.a2sf_prefill_host_workspace_bytes(p, n),), dtype=torch.uint8, device=dev)
+        strides = (w.H * n * d, n * d, d)
+
+        def e2e_step():
+            t0 = time.perf_counter()
+            addr = a2sf.a2sf_prefill_host(p, n, hq, hk, hv, hout, hs, hkept, hws)
+            cache.a2sf_cache_load(addr[0], addr[1], addr[2], addr[3], n=n, strides=strides)
+            torch.cuda.synchronize()
+            t1 = time.perf_counter()
+            for t in range(T):
+                cache.a2sf_decode_step_host(w.alpha, hdq[t], hdk[t], hdv[t], ho, he)
+            t2 = time.perf_counter()
+            return (t1 - t0) * 1e3, (t2 - t1) * 1e3
+
+        ke = max(1, min(args.steps, args.e2e_steps))
+        e2e_step()
+        a2dist.barrier()
+        res = [e2e_step() for _ in range(ke)]
+        a2dist.barrier()
+        e_pre = sum(r[0] for r in res) / ke
+        e_dec = sum(r[1] for r in res) / ke
+        eb = w.elem_bytes
+        h2d = 3 * U * n * d * eb + T * 3 * U * d * eb
+        d2h = U * n * d * eb + U * n * 4 + U * m * 4 + T * (U * d * eb + U * 4)
+        e2e = {"pre_ms": e_pre, "dec_ms": e_dec, "h2d": h2d, "d2h": d2h, "steps": ke}
+
+    # ---- combine over ranks ------------------------------------------------------------
+    bytes_per_launch = U * w.decode_bytes_per_unit_step()
+    flops = w.prefill_flops_per_unit()
+    prefill_flops = U * (flops["pass1"] + flops["pass2"])
+    total_units, max_total_ms = a2dist.job_throughput(U, total_ms, dev)
+    max_decode_ms = a2dist.max_over_ranks(decode_ms, dev)
+    max_prefill_ms = a2dist.max_over_ranks(prefill_ms, dev)
+    max_load_ms = a2dist.max_over_ranks(load_ms, dev)
+    scale_units = total_units / U                      # = world size
+    K = args.steps
+    value = scale_units * bytes_per_launch * T * K / (max_decode_ms * 1e-3) / 1e9
+    prefill_tflops = scale_units * prefill_flops * K / (max_prefill_ms * 1e-3) / 1e12
+    peaks = load_peaks()
+    launch_us = decode_ms / (K * T) * 1e3
+    achieved = bytes_per_launch / (launch_us * 1e-6) / 1e9
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": args.warmup, "ms_per_step": max_total_ms / K, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": {"bf16": "bf16", "fp16": "f16", "fp32": "f32"}[w.dtype],
+        "data": "synthetic",
+        "config": {"workload": f"{w.name} (config {w.index}): B{w.B} H{w.H} d{d} n{n} alpha{w.alpha} "
+                               f"budget{w.budget} recent{w.recent} decode_steps{T} per GPU",
+                   "l2": "inputs_larger_than_l2" if bytes_per_launch > 126e6 else "l2_resident_working_set",
+                   "units_per_gpu": U, "step": "prefill+select+cache_load+decode_steps"},
+        "phases_ms_per_step": {"prefill": max_prefill_ms / K, "cache_load": max_load_ms / K,
+                               "decode": max_decode_ms / K},
+        "prefill": {"metric": "prefill_scoring_tflops", "value": prefill_tflops, "unit": "TFLOP/s",
+                    "flops_per_step": prefill_flops, "frac_of_measured_bf16_sustained":
+                        prefill_tflops / scale_units / peaks["bf16_tflops_sustained"],
+                    "frac_of_nominal_bf16": prefill_tflops / scale_units / NOMINAL["bf16_tflops"]},
+        "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": achieved,
+                     "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                     "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
+                     "traffic": None, "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if e2e is not None:
+        e_dec = a2dist.max_over_ranks(e2e["dec_ms"], dev)
+        e_pre = a2dist.max_over_ranks(e2e["pre_ms"], dev)
+        result["e2e"] = {"value": scale_units * bytes_per_launch * T / (e_dec * 1e-3) / 1e9, "unit": UNIT,
+                         "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                         "ms_per_step": e_pre + e_dec, "prefill_ms": e_pre, "decode_ms": e_dec,
+                         "steps": e2e["steps"]}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(w, T, q, k, v, dq, dk, dv)
+    cache.close()
+    if rank == 0:
+        print(json.dumps(result))
+    a2dist.finalize()
+
+
+def oracle_sample(w, units_sel, dsteps, q, k, v, dq, dk, dv, threads):
+    """Times the oracle, as it stands, on the listed units: prefill + `dsteps` decode steps."""
+    import numpy as np
+
+    import oracle
+
+    ub = [(u // w.H, u % w.H) for u in units_sel]
+    f64 = lambda t: t.detach().cpu().to(torch.float64).numpy()
+    Q = np.stack([f64(q[b, h]) for b, h in ub])
+    K = np.stack([f64(k[b, h]) for b, h in ub])
+    V = np.stack([f64(v[b, h]) for b, h in ub])
+    t0 = time.perf_counter()
+    ref = oracle.prefill(Q, K, V, w.scale, [w.alpha], w.budget, w.recent, nthreads=threads)
+    t1 = time.perf_counter()
+    oc = oracle.Cache(len(ub), w.d, w.budget, w.recent, w.scale)
+    oc.load(K, V, ref["S"][:, 0], ref["kept"])
+    ins = [[np.stack([f64(x[t, b, h]) for b, h in ub]) for x in (dq, dk, dv)] for t in range(dsteps)]
+    t2 = time.perf_counter()
+    for t in range(dsteps):
+        oc.step(*ins[t], w.alpha, nthreads=threads)
+    t3 = time.perf_counter()
+    return t1 - t0, t3 - t2, ref["threads"]
+
+
+def cpu_baseline(w, T, q, k, v, dq, dk, dv):
+    import oracle
+
+    threads = oracle.host_threads()
+    # bounded sample: one unit per host thread; decode steps capped
+    n_units = min(w.units, threads)
+    dsteps = min(T, 64)
+    units_sel = [int(i * (w.units - 1) / max(1, n_units - 1)) for i in range(n_units)] if n_units > 1 else [0]
+    pre_s, dec_s, used = oracle_sample(w, units_sel, dsteps, q, k, v, dq, dk, dv, threads)
+    flops = w.prefill_flops_per_unit()
+    return {"value": n_units * dsteps * w.decode_bytes_per_unit_step() / dec_s / 1e9, "unit": UNIT,
+            "cores": int(used), "kind": "oracle",
+            "sample": f"{n_units} of {w.units} units: prefill n={w.n} ({pre_s:.2f} s) + {dsteps} decode steps "
+                      f"({dec_s:.3f} s), fp64",
+            "prefill_tflops": n_units * (flops["pass1"] + flops["pass2"]) / pre_s / 1e12,
+            "prefill_units_per_s": n_units / pre_s, "decode_unit_steps_per_s": n_units * dsteps / dec_s}
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle on the host cores, a bounded sample per step."""
+    rank, _, world = a2dist.env_world()
+    if rank != 0:
+        return
+    import oracle
+
+    w = wl.WORKLOADS[args.workload]
+    T = args.decode_steps or w.steps
+    threads = oracle.host_threads()
+    n_units = min(w.units, threads)
+    dsteps = min(T, 32)
+    units_sel = [int(i * (w.units - 1) / max(1, n_units - 1)) for i in range(n_units)] if n_units > 1 else [0]
+    bsel = sorted({u // w.H for u in units_sel})
+    # generate only the sampled units' inputs (coordinate-addressed generator)
+    qs, ks, vs, dqs, dks, dvs = {}, {}, {}, {}, {}, {}
+    for u in units_sel:
+        b, h = u // w.H, u % w.H
+        a, b_, c = wl.make_prompt(w, "cpu", (b, b + 1), (h, h + 1))
+        qs[u], ks[u], vs[u] = a[0, 0], b_[0, 0], c[0, 0]
+        a, b_, c = wl.make_decode(w, "cpu", (0, dsteps), (b, b + 1), (h, h + 1))
+        dqs[u], dks[u], dvs[u] = a[:, 0, 0], b_[:, 0, 0], c[:, 0, 0]
+    w1 = w.scaled(B=1, H=n_units)
+    q = torch.stack([qs[u] for u in units_sel])[None]
+    k = torch.stack([ks[u] for u in units_sel])[None]
+    v = torch.stack([vs[u] for u in units_sel])[None]
+    dq = torch.stack([dqs[u] for u in units_sel], 1)[:, None]
+    dk = torch.stack([dks[u] for u in units_sel], 1)[:, None]
+    dv = torch.stack([dvs[u] for u in units_sel], 1)[:, None]
+    sel = list(range(n_units))
+    pre, dec, used = [], [], threads
+    for i in range(args.warmup + args.steps):
+        ps, ds, used = oracle_sample(w1, sel, dsteps, q, k, v, dq, dk, dv, threads)
+        if i >= args.warmup:
+            pre.append(ps)
+            dec.append(ds)
+    K = args.steps
+    value = n_units * dsteps * K * w.decode_bytes_per_unit_step() / sum(dec) / 1e9
+    sample = (f"{n_units} of {w.units} units per step: prefill n={w.n} + {dsteps} of {T} decode steps, fp64 "
+              f"oracle, {used} threads")
+    flops = w.prefill_flops_per_unit()
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": K, "warmup": args.warmup, "ms_per_step": (sum(pre) + sum(dec)) / K * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name} (config {w.index}): B{w.B} H{w.H} d{w.d} n{w.n} alpha{w.alpha} "
+                               f"budget{w.budget} recent{w.recent} decode_steps{T} per GPU",
+                   "sample": sample},
+        "prefill": {"metric": "prefill_scoring_tflops", "unit": "TFLOP/s",
+                    "value": n_units * K * (flops["pass1"] + flops["pass2"]) / sum(pre) / 1e12},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": int(used), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2_13b", choices=sorted(wl.WORKLOADS))
+    ap.add_argument("--decode-steps", type=int, default=0, help="override T (0 = the workload's)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

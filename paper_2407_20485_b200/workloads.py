@@ -223,18 +223,21 @@ def make_prompt(w: Workload, device="cpu",
     return q, k, v
 
 
-def make_prompt_chunked(w: Workload, device, max_units_per_chunk: int = 64):
+def make_prompt_chunked(w: Workload, device, max_units_per_chunk: int = 64,
+                        b_range: Optional[Tuple[int, int]] = None):
     """Full-size prompt tensors generated head-block by head-block so that the
-    float64 intermediates stay small next to the result."""
-    q = torch.empty((w.B, w.H, w.n, w.d), dtype=w.torch_dtype, device=device)
+    float64 intermediates stay small next to the result.  ``b_range`` selects a
+    slice of the batch (one rank's share of a larger job)."""
+    b0, b1 = b_range or (0, w.B)
+    q = torch.empty((b1 - b0, w.H, w.n, w.d), dtype=w.torch_dtype, device=device)
     k = torch.empty_like(q)
     v = torch.empty_like(q)
     hstep = max(1, min(w.H, max_units_per_chunk))
-    for b in range(w.B):
+    for b in range(b0, b1):
         for h0 in range(0, w.H, hstep):
             h1 = min(w.H, h0 + hstep)
             qq, kk, vv = make_prompt(w, device, (b, b + 1), (h0, h1))
-            q[b, h0:h1], k[b, h0:h1], v[b, h0:h1] = qq[0], kk[0], vv[0]
+            q[b - b0, h0:h1], k[b - b0, h0:h1], v[b - b0, h0:h1] = qq[0], kk[0], vv[0]
     return q, k, v
 
 
