@@ -114,6 +114,8 @@ def run_ours(args):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     w = wl.WORKLOADS[args.workload]
+    if args.batch:
+        w = w.scaled(B=args.batch)
     T = args.decode_steps or w.steps
     # weak scaling: every rank owns a full per-GPU batch of a job world x as large
     wg = w.scaled(B=w.B * world, steps=T)
@@ -305,6 +307,8 @@ def run_reference(args):
     import oracle
 
     w = wl.WORKLOADS[args.workload]
+    if args.batch:
+        w = w.scaled(B=args.batch)
     T = args.decode_steps or w.steps
     threads = oracle.host_threads()
     n_units = min(w.units, threads)
@@ -362,6 +366,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_13b", choices=sorted(wl.WORKLOADS))
     ap.add_argument("--decode-steps", type=int, default=0, help="override T (0 = the workload's)")
+    ap.add_argument("--batch", type=int, default=0, help="override the per-GPU batch (0 = the workload's); "
+                    "smaller cases for profiler captures")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
