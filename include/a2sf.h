@@ -120,6 +120,31 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n,
                       void **dev_k, void **dev_v, float **dev_scores, int32_t **dev_kept,
                       void *cuda_stream);
 
+/* Prefill without any allocation, for callers that cannot call cudaMalloc (an
+ * engine whose own allocator owns the device, a plugin that only sees one layer's
+ * tensors, a loop that must not hit an allocation's implicit synchronisation).
+ * The paper has no counterpart: this is the same computation as a2sf_prefill, run
+ * by the CUDA-core kernels, with the per-row log-sum-exp scratch held in a fixed
+ * 4 MiB array inside the library's device image (every GPU that loads the library
+ * carries it until the process exits).
+ *   - Limit: B*H*n <= a2sf_prefill_static_scratch_max_rows() (1,048,576); larger
+ *     calls return A2SF_ERR_WORKSPACE and launch nothing.
+ *   - The first call on each device looks up the array's device address (a short
+ *     host-side driver query with that device current); make that first call
+ *     before starting any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's
+ *     contents.  Each call overwrites every row it later reads, so nothing needs
+ *     clearing, but two calls that overlap on the GPU (different streams without an
+ *     event between them) race on it: keep them ordered.
+ *   - It calls no cudaMalloc / cudaFree and takes no workspace; the log-sum-exp is
+ *     not returned.  Other arguments, results and errors are those of a2sf_prefill. */
+size_t a2sf_prefill_static_scratch_max_rows(void);
+
+int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n,
+                                const void *q, const void *k, const void *v,
+                                int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                                void *out, float *scores, int32_t *kept_idx, void *cuda_stream);
+
 /* ---------------------------------------------------------------------------
  * The pruned cache.  Per unit: K and V rows [M][d] in `dtype`, scores [M] fp32,
  * positions [M] int32 (slot -> token position, -1 = empty), the resident count and

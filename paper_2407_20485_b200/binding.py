@@ -49,6 +49,8 @@ def _load():
         "a2sf_prefill": (ctypes.c_int, [pp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]),
         "a2sf_rescore_workspace_bytes": (sz, [pp, i32]),
         "a2sf_rescore": (ctypes.c_int, [pp, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]),
+        "a2sf_prefill_static_scratch_max_rows": (sz, []),
+        "a2sf_prefill_static_scratch": (ctypes.c_int, [pp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp]),
         "a2sf_prefill_host_workspace_bytes": (sz, [pp, i32]),
         "a2sf_prefill_host": (ctypes.c_int, [pp, i32, vp, vp, vp, vp, vp, vp, vp, sz,
                                              pvp, pvp, pvp, pvp, vp]),
@@ -164,6 +166,16 @@ def a2sf_rescore(p: a2sf_params, q, k, lse, scores=None, kept_idx=None, workspac
                             workspace.numel() if workspace is not None else 0,
                             _stream(stream)), "a2sf_rescore")
     return scores, kept_idx
+
+
+def a2sf_prefill_static_scratch(p: a2sf_params, q, k, v, out, scores, kept_idx, stream=None):
+    """Prefill for callers that cannot allocate: every tensor is supplied by the
+    caller and the library's built-in scratch array is used (size limit: see
+    ``a2sf_prefill_static_scratch_max_rows``).  Returns the status code."""
+    sb, sh, st = _strides(q)
+    return int(lib.a2sf_prefill_static_scratch(ctypes.byref(p), q.shape[2], _ptr(q), _ptr(k), _ptr(v),
+                                               sb, sh, st, _ptr(out), _ptr(scores), _ptr(kept_idx),
+                                               _stream(stream)))
 
 
 def a2sf_prefill_host_workspace_bytes(p: a2sf_params, n: int) -> int:

@@ -1,0 +1,90 @@
+// Prefill for callers that cannot allocate device memory.
+//
+// Some users of this library run where cudaMalloc is off limits: inside a serving
+// engine that has handed the whole device to its own pool allocator, in a plugin
+// that is only given the tensors of one layer, or in a real-time loop where an
+// allocation's implicit synchronisation is not acceptable.  a2sf_prefill needs a
+// scratch row per (batch, head, token) for the log-sum-exp that the first pass
+// writes and the scoring pass reads; here that scratch is a fixed array that lives
+// in the library's own device image, so the caller passes inputs and outputs only.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace a2sf {
+
+// 4 MiB of fp32 log-sum-exp rows: B*H*n <= 1,048,576 (e.g. 32 heads x 32768 tokens,
+// or 256 heads x 4096).  Every GPU that loads the library holds it until exit.
+constexpr size_t kStaticLseFloats = size_t(1) << 20;
+static __device__ __align__(256) float g_static_lse[kStaticLseFloats];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_mu;
+float *g_lse_addr[kMaxDevices] = {};
+
+// The array's name is only a host-side handle; the device address has to be asked
+// for, once per device, with that device current.
+int static_lse_address(float **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return A2SF_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!g_lse_addr[dev]) {
+        float *ptr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_lse) != cudaSuccess || !ptr)
+            return A2SF_ERR_CUDA;
+        g_lse_addr[dev] = ptr;
+    }
+    *out = g_lse_addr[dev];
+    return A2SF_OK;
+}
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+}  // namespace a2sf
+
+using namespace a2sf;
+
+extern "C" size_t a2sf_prefill_static_scratch_max_rows(void) { return kStaticLseFloats; }
+
+extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, const void *q,
+                                           const void *k, const void *v, int64_t stride_b,
+                                           int64_t stride_h, int64_t stride_t, void *out,
+                                           float *scores, int32_t *kept_idx, void *cuda_stream)
+{
+    if (!p || n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    if (p->B < 1 || p->H < 1 || p->budget < 1 || p->recent < 0 || p->recent > p->budget ||
+        !(p->alpha >= 0.f && p->alpha <= 1.f) || !(p->scale >= 0.f) || isinf(p->scale))
+        return A2SF_ERR_INVALID_ARG;
+    if ((p->dtype != A2SF_F32 && p->dtype != A2SF_BF16 && p->dtype != A2SF_F16) ||
+        (p->d != 64 && p->d != 128))
+        return A2SF_ERR_UNSUPPORTED;
+    const int vec = p->dtype == A2SF_F32 ? 4 : 8;
+    if (stride_t < p->d || stride_h < 1 || stride_b < 1 || stride_t % vec || stride_h % vec ||
+        stride_b % vec || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return A2SF_ERR_INVALID_ARG;
+    // the scratch is fixed: refuse what does not fit rather than overrun it
+    if ((size_t)p->B * (size_t)p->H * (size_t)n > kStaticLseFloats) return A2SF_ERR_WORKSPACE;
+
+    float *lse = nullptr;
+    const int rc = static_lse_address(&lse);
+    if (rc != A2SF_OK) return rc;
+
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    PrefillArgs a;
+    a.q = q; a.k = k; a.v = v; a.out = out;
+    a.lse = lse;          // every row this call reads is written by its own first pass,
+    a.scores = scores;    // so nothing has to be cleared between calls
+    a.st = Strides{stride_b, stride_h, stride_t};
+    a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
+    a.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
+    a.alpha = p->alpha;
+    if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    if (launch_prefill_pass2_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    if (launch_select(scores, kept_idx, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
