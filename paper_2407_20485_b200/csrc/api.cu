@@ -52,7 +52,9 @@ static size_t prefill_ws_bytes(const a2sf_params *p, int n)
 static int run_scores_and_select(const a2sf_params *p, int n, PrefillArgs &a, int32_t *kept,
                                  cudaStream_t s)
 {
-    if (launch_prefill_pass2_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    const cudaError_t e2 = prefill_tc_supported(p->dtype, a) ? launch_prefill_pass2_tc(p->dtype, a, s)
+                                                             : launch_prefill_pass2_simt(p->dtype, a, s);
+    if (e2 != cudaSuccess) return A2SF_ERR_CUDA;
     if (launch_select(a.scores, kept, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
         return A2SF_ERR_CUDA;
     return A2SF_OK;
@@ -363,9 +365,7 @@ int64_t a2sf_kernel_launch_count(void) { return g_launches.load(std::memory_orde
 
 int a2sf_last_device_status(void *cuda_stream)
 {
-    if (cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
-        return A2SF_ERR_CUDA;
-    return A2SF_OK;
+    return read_and_clear_tc_status(static_cast<cudaStream_t>(cuda_stream));
 }
 
 const char *a2sf_status_string(int status)

@@ -110,6 +110,11 @@ struct PrefillArgs {
 cudaError_t launch_prefill_pass1_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
 cudaError_t launch_prefill_pass2_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
 
+// tensor-core path (16-bit storage, d = 128)
+bool prefill_tc_supported(int dtype, const PrefillArgs &a);
+cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
+int read_and_clear_tc_status(cudaStream_t s);
+
 cudaError_t launch_select(const float *scores, int32_t *kept, int U, int n, int M, int R,
                           cudaStream_t s);
 
