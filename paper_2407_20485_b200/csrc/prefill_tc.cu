@@ -247,7 +247,7 @@ bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillA
 bool prefill_tc_supported(int dtype, const PrefillArgs &a)
 {
     return (dtype == A2SF_BF16 || dtype == A2SF_F16) && a.d == kD &&
-           (a.n + kBlk - 1) / kBlk <= 65535 && encode_fn() != nullptr;
+           (a.n + kBlk - 1) / kBlk <= 65535;
 }
 
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
