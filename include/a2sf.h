@@ -213,7 +213,9 @@ int a2sf_cache_import(a2sf_cache *cache, const void *k, const void *v, const flo
 int64_t a2sf_kernel_launch_count(void);
 
 /* Synchronises the stream and returns the sticky device-side status (A2SF_OK, or
- * A2SF_ERR_TIMEOUT if a kernel abandoned a bounded wait), then clears it. */
+ * A2SF_ERR_TIMEOUT if a kernel abandoned a bounded wait), then clears it.  While the
+ * status is set the tensor-core prefill kernels return without working, so results
+ * of calls made after a timeout and before this call are undefined. */
 int a2sf_last_device_status(void *cuda_stream);
 
 const char *a2sf_status_string(int status);

@@ -112,7 +112,9 @@ int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, 
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha;
-    if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    const cudaError_t e1 = prefill_tc_supported(p->dtype, a) ? launch_prefill_pass1_tc(p->dtype, a, s)
+                                                             : launch_prefill_pass1_simt(p->dtype, a, s);
+    if (e1 != cudaSuccess) return A2SF_ERR_CUDA;
     return run_scores_and_select(p, n, a, kept_idx, s);
 }
 

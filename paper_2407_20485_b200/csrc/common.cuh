@@ -112,6 +112,7 @@ cudaError_t launch_prefill_pass2_simt(int dtype, const PrefillArgs &a, cudaStrea
 
 // tensor-core path (16-bit storage, d = 128)
 bool prefill_tc_supported(int dtype, const PrefillArgs &a);
+cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 int read_and_clear_tc_status(cudaStream_t s);
 

@@ -9,6 +9,7 @@
 // Warp roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and
 // TMEM owner, warps 2-5 = epilogue (one TMEM lane quarter each).
 #include <mutex>
+#include <type_traits>
 
 #include "common.cuh"
 #include "tc_sm100.cuh"
@@ -71,6 +72,12 @@ __global__ void __launch_bounds__(kScoreThreads)
 score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
               ScoreArgs a, int ab_fmt)
 {
+    // once any CTA has given up on a wait, the rest of the grid drains without working
+    __shared__ int s_skip;
+    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int *>(&g_tc_status);
+    __syncthreads();
+    if (s_skip) return;
+
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                 ~uintptr_t(1023));
@@ -205,6 +212,302 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
     if (threadIdx.x == 0 && sh->abort_flag) g_tc_status = A2SF_ERR_TIMEOUT;
 }
 
+
+// ============================================================================================
+// Attention pass (paper Eq. 3: causal softmax attention):  out_i = sum_j P_ij v_j,  lse_i.
+//
+// One CTA owns 128 query rows (TMEM lanes) and walks the key tiles up to the diagonal.
+//   S = Q K^T          -> TMEM (two buffers, so the next tile's logits are computed while the
+//                         current tile is in the softmax warps)
+//   softmax warps      : one thread per row; running maximum kept lazily (the accumulator is
+//                         rescaled only when the maximum grows by more than 2^8), P rounded to
+//                         the storage type and written to shared memory in the 128-byte-swizzled
+//                         K-major layout the MMA reads; the row sum uses the unrounded values
+//   O += P V           -> TMEM; V is consumed as an MN-major operand straight from its TMA tile
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
+// softmax + epilogue.
+// ============================================================================================
+constexpr int kAttnThreads = 192;
+constexpr int kKvStages = 2;
+constexpr float kRescaleThreshold = 8.0f;     // log2 units
+
+struct AttnArgs {
+    void *out;            // [B][H][n][d], strides below
+    float *lse;           // [U][n]
+    int64_t st_b, st_h, st_t;
+    int n, H;
+    float sl2;            // scale * log2(e)
+};
+
+struct AttnShared {
+    uint64_t q_full, k_full[kKvStages], k_empty[kKvStages], v_full[kKvStages], v_empty[kKvStages];
+    uint64_t s_full[2], s_empty[2], p_full, p_empty;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// Q, K ring, V ring, P
+constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (2 + 2 * kKvStages) + sizeof(AttnShared);
+
+template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
+template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b)
+{
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kAttnThreads)
+attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+             const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
+{
+    // once any CTA has given up on a wait, the rest of the grid drains without working
+    __shared__ int s_skip;
+    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int *>(&g_tc_status);
+    __syncthreads();
+    if (s_skip) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                ~uintptr_t(1023));
+    uint8_t *Qs = smem;
+    uint8_t *Ps = smem + kTileBytes;
+    uint8_t *Ks = smem + 2 * kTileBytes;
+    uint8_t *Vs = Ks + kKvStages * kTileBytes;
+    AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kKvStages * kTileBytes);
+
+    constexpr int ab_fmt = sizeof(T) == 2 && std::is_same<T, __nv_bfloat16>::value ? 1 : 0;
+    const int u = blockIdx.x;
+    const int T_total = (a.n + kBlk - 1) / kBlk;
+    const int rb = T_total - 1 - blockIdx.y;            // longest rows first
+    const int nt = rb + 1;                              // key tiles 0 .. rb
+    const int b = u / a.H, h = u % a.H;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int *abort_flag = &sh->abort_flag;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&sh->q_full, 1);
+        for (int s = 0; s < kKvStages; ++s) {
+            mbar_init(&sh->k_full[s], 1); mbar_init(&sh->k_empty[s], 1);
+            mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1);
+        }
+        for (int x = 0; x < 2; ++x) { mbar_init(&sh->s_full[x], 1); mbar_init(&sh->s_empty[x], kBlk); }
+        mbar_init(&sh->p_full, kBlk);
+        mbar_init(&sh->p_empty, 1);
+        sh->abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(&sh->tmem_base, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sh->tmem_base;
+    const uint32_t tmem_o = tmem_base + 2 * kBlk;        // S0 | S1 | O
+
+    if (warp == 0) {
+        // ---- TMA producer -------------------------------------------------------------
+        if (lane == 0) {
+            prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+            mbar_arrive_expect_tx(&sh->q_full, kTileBytes);
+            tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rb * kBlk, h, b);
+            tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rb * kBlk, h, b);
+            int issued = 0;
+            for (int t = 0; t < nt; ++t) {
+                const int s = t % kKvStages;
+                const uint32_t ph = (t / kKvStages) & 1;
+                if (!mbar_wait(&sh->k_empty[s], ph ^ 1, abort_flag)) break;
+                mbar_arrive_expect_tx(&sh->k_full[s], kTileBytes);
+                tma_load_4d(Ks + s * kTileBytes, &tmap_k, &sh->k_full[s], 0, t * kBlk, h, b);
+                tma_load_4d(Ks + s * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[s], 64, t * kBlk, h, b);
+                if (!mbar_wait(&sh->v_empty[s], ph ^ 1, abort_flag)) { issued = -(t + 1); break; }
+                mbar_arrive_expect_tx(&sh->v_full[s], kTileBytes);
+                tma_load_4d(Vs + s * kTileBytes, &tmap_v, &sh->v_full[s], 0, t * kBlk, h, b);
+                tma_load_4d(Vs + s * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[s], 64, t * kBlk, h, b);
+                issued = t + 1;
+            }
+            if (*abort_flag) {
+                // bounded chance for copies in flight to land before the CTA exits
+                int dummy = 0;
+                const int kdone = issued < 0 ? -issued : issued;
+                const int vdone = issued < 0 ? -issued - 1 : issued;
+                for (int t = max(0, kdone - kKvStages); t < kdone; ++t)
+                    mbar_wait(&sh->k_full[t % kKvStages], (t / kKvStages) & 1, &dummy);
+                for (int t = max(0, vdone - kKvStages); t < vdone; ++t)
+                    mbar_wait(&sh->v_full[t % kKvStages], (t / kKvStages) & 1, &dummy);
+                mbar_wait(&sh->q_full, 0, &dummy);
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer -----------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
+            const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
+            const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps);
+            auto issue_s = [&](int t) -> bool {
+                const int s = t % kKvStages;
+                const int sb = t & 1;
+                if (!mbar_wait(&sh->k_full[s], (t / kKvStages) & 1, abort_flag)) return false;
+                if (!mbar_wait(&sh->s_empty[sb], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
+                tc_fence_after_sync();
+                issue_qk_mma(tmem_base + sb * kBlk, q_addr, smem_u32(Ks + s * kTileBytes), idesc_qk);
+                umma_commit(&sh->k_empty[s]);
+                umma_commit(&sh->s_full[sb]);
+                return true;
+            };
+            bool ok = mbar_wait(&sh->q_full, 0, abort_flag);
+            ok = ok && issue_s(0);
+            for (int t = 0; ok && t < nt; ++t) {
+                if (t + 1 < nt && !issue_s(t + 1)) break;
+                const int s = t % kKvStages;
+                if (!mbar_wait(&sh->p_full, t & 1, abort_flag)) break;
+                if (!mbar_wait(&sh->v_full[s], (t / kKvStages) & 1, abort_flag)) break;
+                tc_fence_after_sync();
+                const uint32_t v_addr = smem_u32(Vs + s * kTileBytes);
+#pragma unroll
+                for (int k = 0; k < kBlk / 16; ++k) {
+                    // A = P: 16 keys = 32 bytes along the swizzled row; B = V: 16 keys = two
+                    // 8-row groups of 1024 bytes, the two 64-wide d halves 16 KB apart
+                    const uint64_t adesc =
+                        make_sdesc_sw128(p_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+                    const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
+                    umma_ss(tmem_o, adesc, bdesc, idesc_pv, (t > 0) || (k > 0));
+                }
+                umma_commit(&sh->v_empty[s]);
+                umma_commit(&sh->p_empty);
+            }
+        }
+    } else {
+        // ---- softmax + epilogue: one thread per query row ------------------------------
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
+        const int i = rb * kBlk + r;
+        const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+        float m_used = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int t = 0; ok && t < nt; ++t) {
+            const int sb = t & 1;
+            if (!mbar_wait(&sh->s_full[sb], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t s_addr = tmem_base + sb * kBlk + lane_off;
+            const bool diag = (t == nt - 1);
+            // pass A: row maximum of the scaled logits (log2 domain)
+            float tmax = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < kBlk / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_wait_ld();
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    float sv = __uint_as_float(v[x]) * a.sl2;
+                    if (diag && c * 32 + x > r) sv = -INFINITY;        // causal mask
+                    tmax = fmaxf(tmax, sv);
+                }
+            }
+            // lazy maximum: keep the old reference unless the new maximum exceeds it by 2^8
+            float factor = 1.f;
+            bool grow = false;
+            if (t == 0) {
+                m_used = tmax;
+            } else if (tmax > m_used + kRescaleThreshold) {
+                factor = ex2_approx(m_used - tmax);
+                m_used = tmax;
+                grow = true;
+            }
+            // P(t-1) has been consumed and O holds tiles 0..t-1 once p_empty completes
+            if (t > 0 && !mbar_wait(&sh->p_empty, (t - 1) & 1, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            if (__any_sync(0xffffffffu, grow)) {
+                l *= factor;
+#pragma unroll 1
+                for (int c = 0; c < kD / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_o + lane_off + c * 32, v);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * factor);
+                    tmem_st32(tmem_o + lane_off + c * 32, v);
+                }
+                tmem_wait_st();
+            }
+            // pass B: probabilities, row sum (unrounded), P tile to shared memory
+            float rowsum = 0.f;
+            const float neg_m = -m_used;
+#pragma unroll 1
+            for (int c = 0; c < kBlk / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(s_addr + c * 32, v);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int x = 0; x < 32; x += 2) {
+                    float p0 = ex2_approx(fmaf(__uint_as_float(v[x]), a.sl2, neg_m));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(v[x + 1]), a.sl2, neg_m));
+                    if (diag) {
+                        if (c * 32 + x > r) p0 = 0.f;
+                        if (c * 32 + x + 1 > r) p1 = 0.f;
+                    }
+                    rowsum += p0 + p1;
+                    pk[x >> 1] = pack2<T>(p0, p1);
+                }
+                // columns c*32 .. c*32+31 = 16-byte chunks (c&1)*4 .. +3 of half c>>1
+                uint8_t *rowp = Ps + (c >> 1) * kHalfBytes + r * 128;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int chunk = ((c & 1) * 4 + q4) ^ (r & 7);
+                    *reinterpret_cast<uint4 *>(rowp + chunk * 16) =
+                        make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+                }
+            }
+            l += rowsum;
+            tc_fence_before_sync();
+            mbar_arrive(&sh->s_empty[sb]);            // the logits buffer may be overwritten
+            fence_async_smem();                       // P stores -> visible to the tensor core
+            mbar_arrive(&sh->p_full);
+        }
+        // ---- epilogue ---------------------------------------------------------------------
+        if (ok && mbar_wait(&sh->p_empty, (nt - 1) & 1, abort_flag)) {
+            tc_fence_after_sync();
+            const float inv = 1.f / l;
+            T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t;
+#pragma unroll 1
+            for (int c = 0; c < kD / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_o + lane_off + c * 32, v);
+                tmem_wait_ld();
+                if (i < a.n) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+                            w[e] = pack2<T>(__uint_as_float(v[q4 * 8 + 2 * e]) * inv,
+                                            __uint_as_float(v[q4 * 8 + 2 * e + 1]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+            if (i < a.n) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+    if (threadIdx.x == 0 && sh->abort_flag) g_tc_status = A2SF_ERR_TIMEOUT;
+}
+
 // ---- host: tensor maps -----------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -248,6 +551,36 @@ bool prefill_tc_supported(int dtype, const PrefillArgs &a)
 {
     return (dtype == A2SF_BF16 || dtype == A2SF_F16) && a.d == kD &&
            (a.n + kBlk - 1) / kBlk <= 65535;
+}
+
+cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
+{
+    CUtensorMap mq, mk, mv;
+    if (!make_tile_map(&mq, dtype, a.q, a) || !make_tile_map(&mk, dtype, a.k, a) ||
+        !make_tile_map(&mv, dtype, a.v, a))
+        return cudaErrorInvalidValue;
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_pass_tc<__half>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return attr_err;
+    AttnArgs aa;
+    aa.out = a.out; aa.lse = a.lse;
+    aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
+    aa.n = a.n; aa.H = a.H;
+    aa.sl2 = a.scale * kLog2e;
+    dim3 grid(a.B * a.H, (a.n + kBlk - 1) / kBlk);
+    if (dtype == A2SF_BF16)
+        attn_pass_tc<__nv_bfloat16><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+    else
+        attn_pass_tc<__half><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+    count_launch();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
