@@ -246,8 +246,8 @@ struct AttnShared {
     int abort_flag;
 };
 
-// Q, K ring, V ring, P
-constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (2 + 2 * kKvStages) + sizeof(AttnShared);
+// Q, P (high part), P (low part, bf16 only), K ring, V ring
+constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (3 + 2 * kKvStages) + sizeof(AttnShared);
 
 template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
 template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b)
@@ -277,11 +277,17 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                                                 ~uintptr_t(1023));
     uint8_t *Qs = smem;
     uint8_t *Ps = smem + kTileBytes;
-    uint8_t *Ks = smem + 2 * kTileBytes;
+    uint8_t *Pl = smem + 2 * kTileBytes;
+    uint8_t *Ks = smem + 3 * kTileBytes;
     uint8_t *Vs = Ks + kKvStages * kTileBytes;
     AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kKvStages * kTileBytes);
 
-    constexpr int ab_fmt = sizeof(T) == 2 && std::is_same<T, __nv_bfloat16>::value ? 1 : 0;
+    constexpr int ab_fmt = std::is_same<T, __nv_bfloat16>::value ? 1 : 0;
+    // A bf16 probability keeps 8 significand bits; where the products p*v cancel, that
+    // rounding alone exceeds the output tolerance.  For bf16 the probabilities are therefore
+    // split into two bf16 terms (p = hi + lo, |lo| <= 2^-9 |hi|) and both are multiplied
+    // with V.  fp16 keeps 11 bits and needs no second term.
+    constexpr bool kSplitP = std::is_same<T, __nv_bfloat16>::value;
     const int u = blockIdx.x;
     const int T_total = (a.n + kBlk - 1) / kBlk;
     const int rb = T_total - 1 - blockIdx.y;            // longest rows first
@@ -350,7 +356,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
             const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
-            const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps);
+            const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps), pl_addr = smem_u32(Pl);
             auto issue_s = [&](int t) -> bool {
                 const int s = t % kKvStages;
                 const int sb = t & 1;
@@ -379,6 +385,15 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                         make_sdesc_sw128(p_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
                     const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
                     umma_ss(tmem_o, adesc, bdesc, idesc_pv, (t > 0) || (k > 0));
+                }
+                if (kSplitP) {
+#pragma unroll
+                    for (int k = 0; k < kBlk / 16; ++k) {
+                        const uint64_t adesc =
+                            make_sdesc_sw128(pl_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+                        const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
+                        umma_ss(tmem_o, adesc, bdesc, idesc_pv, 1);
+                    }
                 }
                 umma_commit(&sh->v_empty[s]);
                 umma_commit(&sh->p_empty);
@@ -446,7 +461,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 uint32_t v[32];
                 tmem_ld32(s_addr + c * 32, v);
                 tmem_wait_ld();
-                uint32_t pk[16];
+                uint32_t pk[16], pl[16];
 #pragma unroll
                 for (int x = 0; x < 32; x += 2) {
                     float p0 = ex2_approx(fmaf(__uint_as_float(v[x]), a.sl2, neg_m));
@@ -456,15 +471,22 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                         if (c * 32 + x + 1 > r) p1 = 0.f;
                     }
                     rowsum += p0 + p1;
-                    pk[x >> 1] = pack2<T>(p0, p1);
+                    const uint32_t hi = pack2<T>(p0, p1);
+                    pk[x >> 1] = hi;
+                    if (kSplitP)      // a bf16 is the upper half of an fp32
+                        pl[x >> 1] = pack2<T>(p0 - __uint_as_float(hi << 16),
+                                              p1 - __uint_as_float(hi & 0xffff0000u));
                 }
                 // columns c*32 .. c*32+31 = 16-byte chunks (c&1)*4 .. +3 of half c>>1
-                uint8_t *rowp = Ps + (c >> 1) * kHalfBytes + r * 128;
+                const int row_off = (c >> 1) * kHalfBytes + r * 128;
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     const int chunk = ((c & 1) * 4 + q4) ^ (r & 7);
-                    *reinterpret_cast<uint4 *>(rowp + chunk * 16) =
+                    *reinterpret_cast<uint4 *>(Ps + row_off + chunk * 16) =
                         make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+                    if (kSplitP)
+                        *reinterpret_cast<uint4 *>(Pl + row_off + chunk * 16) =
+                            make_uint4(pl[q4 * 4], pl[q4 * 4 + 1], pl[q4 * 4 + 2], pl[q4 * 4 + 3]);
                 }
             }
             l += rowsum;
