@@ -367,7 +367,9 @@ int64_t a2sf_kernel_launch_count(void) { return g_launches.load(std::memory_orde
 
 int a2sf_last_device_status(void *cuda_stream)
 {
-    return read_and_clear_tc_status(static_cast<cudaStream_t>(cuda_stream));
+    const int a = read_and_clear_tc_status(static_cast<cudaStream_t>(cuda_stream));
+    const int b = read_and_clear_decode_status(static_cast<cudaStream_t>(cuda_stream));
+    return a != A2SF_OK ? a : b;
 }
 
 const char *a2sf_status_string(int status)

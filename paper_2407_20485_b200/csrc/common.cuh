@@ -135,4 +135,6 @@ cudaError_t launch_cache_load(const CacheView &c, int H, int n, const void *k, c
 cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
                                const void *v_new, void *out, int32_t *evicted, cudaStream_t s);
 
+int read_and_clear_decode_status(cudaStream_t s);
+
 }  // namespace a2sf

@@ -6,10 +6,24 @@
 // Memory-bound: every K and V row of the head is read exactly once with 16-byte
 // loads, lanes laid across the row so a warp reads whole 512-byte spans.
 #include "common.cuh"
+#include "tc_sm100.cuh"
 
 namespace a2sf {
 
+// sticky device-side status of the decode kernels (a bounded wait that ran out)
+static __device__ int g_decode_status = 0;
+
 namespace {
+
+int *decode_status_word()
+{
+    static int *ptr = nullptr;
+    if (!ptr) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_decode_status) == cudaSuccess) ptr = static_cast<int *>(p);
+    }
+    return ptr;
+}
 
 constexpr int kDecodeThreads = 256;
 constexpr int kUnroll = 4;
@@ -213,6 +227,298 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
     }
 }
 
+
+// ============================================================================================
+// Streaming variant: persistent CTAs, K/V rows brought into a shared-memory ring by bulk
+// asynchronous copies that a producer warp keeps issuing across phase and unit boundaries,
+// so HBM requests stay in flight while the consumer warps sit in the softmax reductions or
+// in the eviction epilogue of the previous head.
+// ============================================================================================
+constexpr int kStreamConsumerWarps = 8;
+constexpr int kStreamConsumers = kStreamConsumerWarps * 32;
+constexpr int kStreamThreads = kStreamConsumers + 32;
+constexpr int kChunkBytes = 16384;
+constexpr int kStreamStages = 10;
+
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        :
+        : "r"(tc::smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(tc::smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void consumer_barrier()
+{
+    tc::named_barrier(1, kStreamConsumers);
+}
+
+__device__ __forceinline__ float consumer_max(float v, float *red)
+{
+    v = warp_max(v);
+    consumer_barrier();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    consumer_barrier();
+    float r = red[0];
+#pragma unroll
+    for (int w = 1; w < kStreamConsumerWarps; ++w) r = fmaxf(r, red[w]);
+    return r;
+}
+
+__device__ __forceinline__ float consumer_sum(float v, float *red)
+{
+    v = warp_sum(v);
+    consumer_barrier();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    consumer_barrier();
+    float r = red[0];
+#pragma unroll
+    for (int w = 1; w < kStreamConsumerWarps; ++w) r += red[w];   // fixed order
+    return r;
+}
+
+struct StreamShared {
+    uint64_t full[kStreamStages], empty[kStreamStages];
+    unsigned long long red_key[kStreamConsumerWarps];
+    float red[kStreamConsumerWarps];
+    int target;
+    int abort_flag;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kStreamThreads)
+decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
+                          const T *__restrict__ k_new, const T *__restrict__ v_new,
+                          T *__restrict__ out, int32_t *__restrict__ evicted, int *status)
+{
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int LPR = D / VEC;                    // lanes per row
+    constexpr int RPW = 32 / LPR;                   // rows per warp-wide 512-byte read
+    constexpr int ROWB = D * (int)sizeof(T);
+    constexpr int CR = kChunkBytes / ROWB;          // rows per chunk
+    constexpr int NW = kStreamConsumerWarps;
+    constexpr int LPC = CR / RPW / NW;              // warp-wide reads per warp and chunk
+    static_assert(LPC == 4, "chunk geometry");
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    const int M = c.M;
+    float *w = reinterpret_cast<float *>(ring + kStreamStages * kChunkBytes);   // [M+1]
+    float *part = w + ((M + 1 + 3) & ~3);                                       // [NW][D]
+    StreamShared *sh = reinterpret_cast<StreamShared *>(part + NW * D);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    volatile int *abort_flag = &sh->abort_flag;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStreamStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], NW); }
+        sh->abort_flag = 0;
+        tc::fence_mbar_init();
+    }
+    __syncthreads();
+
+    // a wait that fails poisons the CTA: every later wait returns at once, control flow stays
+    // uniform (all consumers still meet at their barriers) and the status word reports it
+    auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
+        if (*abort_flag) return false;
+        return tc::mbar_wait(bar, parity, abort_flag);
+    };
+
+    if (warp == NW) {
+        // ---- producer: one lane streams K then V of every unit this CTA owns ----------------
+        if (lane == 0) {
+            uint32_t g = 0;                         // chunk sequence number (same on both sides)
+            uint32_t inflight_from = 0;
+            bool alive = true;
+            for (int u = blockIdx.x; alive && u < c.U; u += gridDim.x) {
+                const int cnt = min(c.count[u], M);
+                for (int pass = 0; alive && pass < 2; ++pass) {
+                    const uint8_t *base = static_cast<const uint8_t *>(pass == 0 ? c.K : c.V) +
+                                          (size_t)u * M * ROWB;
+                    for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
+                        const int s = g % kStreamStages;
+                        if (!wait(&sh->empty[s], ((g / kStreamStages) & 1) ^ 1)) { alive = false; break; }
+                        const uint32_t bytes = (uint32_t)min(CR, cnt - r0) * ROWB;
+                        tc::mbar_arrive_expect_tx(&sh->full[s], bytes);
+                        bulk_load(ring + s * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[s]);
+                    }
+                }
+            }
+            if (!alive) {
+                // bounded chance for copies already issued to land before the CTA exits
+                int dummy = 0;
+                inflight_from = g > (uint32_t)kStreamStages ? g - kStreamStages : 0;
+                for (uint32_t x = inflight_from; x < g; ++x)
+                    tc::mbar_wait(&sh->full[x % kStreamStages], (x / kStreamStages) & 1, &dummy);
+            }
+        }
+    } else {
+        // ---- consumers ---------------------------------------------------------------------
+        const int sub = lane % LPR, rsel = lane / LPR;
+        uint32_t g = 0;
+        for (int u = blockIdx.x; u < c.U; u += gridDim.x) {
+            const int cnt = min(c.count[u], M);
+            const int p = c.len[u];
+            T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
+            T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
+            float *Su = c.S + (size_t)u * M;
+            int32_t *posu = c.pos + (size_t)u * M;
+
+            float qf[VEC];
+            Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
+
+            // (i) logits
+            for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
+                const int s = g % kStreamStages;
+                wait(&sh->full[s], (g / kStreamStages) & 1);
+                const uint8_t *stage = ring + s * kChunkBytes;
+                uint4 r[LPC];
+#pragma unroll
+                for (int x = 0; x < LPC; ++x) {
+                    const int lrow = (x * NW + warp) * RPW + rsel;
+                    r[x] = *reinterpret_cast<const uint4 *>(stage + lrow * ROWB + sub * 16);
+                }
+#pragma unroll
+                for (int x = 0; x < LPC; ++x) {
+                    const int row = r0 + (x * NW + warp) * RPW + rsel;
+                    float kf[VEC];
+                    Elem<T>::unpack(r[x], kf);
+                    float dot = 0.f;
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    if (sub == 0 && row < cnt) w[row] = dot * c.scale;
+                }
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+            }
+            if (warp == 0) {
+                float kf[VEC];
+                Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC), kf);
+                float dot = 0.f;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
+#pragma unroll
+                for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                if (lane == 0) w[cnt] = dot * c.scale;
+            }
+            consumer_barrier();
+
+            // (ii) softmax over resident + self
+            float m = -INFINITY;
+            for (int s_ = tid; s_ <= cnt; s_ += kStreamConsumers) m = fmaxf(m, w[s_]);
+            m = consumer_max(m, sh->red);
+            float l = 0.f;
+            for (int s_ = tid; s_ <= cnt; s_ += kStreamConsumers) {
+                const float e = expf(w[s_] - m);
+                w[s_] = e;
+                l += e;
+            }
+            l = consumer_sum(l, sh->red);
+            const float e_self = w[cnt];
+
+            // (iii) out
+            float acc[VEC];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+            for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
+                const int s = g % kStreamStages;
+                wait(&sh->full[s], (g / kStreamStages) & 1);
+                const uint8_t *stage = ring + s * kChunkBytes;
+                uint4 r[LPC];
+#pragma unroll
+                for (int x = 0; x < LPC; ++x) {
+                    const int lrow = (x * NW + warp) * RPW + rsel;
+                    r[x] = *reinterpret_cast<const uint4 *>(stage + lrow * ROWB + sub * 16);
+                }
+#pragma unroll
+                for (int x = 0; x < LPC; ++x) {
+                    const int row = r0 + (x * NW + warp) * RPW + rsel;
+                    if (row < cnt) {                 // rows past the count hold stale bytes
+                        const float ws = w[row];
+                        float vf[VEC];
+                        Elem<T>::unpack(r[x], vf);
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) acc[e] = fmaf(ws, vf[e], acc[e]);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+            }
+#pragma unroll
+            for (int o = LPR; o < 32; o <<= 1)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+            if (rsel == 0)
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) part[warp * D + sub * VEC + e] = acc[e];
+            consumer_barrier();
+            if (tid < D) {
+                float o = 0.f;
+#pragma unroll
+                for (int x = 0; x < NW; ++x) o += part[x * D + tid];
+                o = fmaf(e_self, Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+                out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
+            }
+
+            // (iv) S <- alpha*S + a ; (v) argmin over the non-recent slots
+            const bool full = cnt >= M;
+            const int newest_evictable = p - c.R;
+            unsigned long long best = ~0ull;
+            int best_slot = -1;
+            for (int s_ = tid; s_ < cnt; s_ += kStreamConsumers) {
+                const float a = w[s_] / l;
+                const float sn = fmaf(alpha, Su[s_], a);
+                Su[s_] = sn;
+                const int ps = posu[s_];
+                if (full && ps <= newest_evictable) {
+                    const unsigned long long key =
+                        ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
+                    if (key < best) { best = key; best_slot = s_; }
+                }
+            }
+            const float a_self = e_self / l;
+            const unsigned long long wbest = warp_min_u64(best);
+            if (lane == 0) sh->red_key[warp] = wbest;
+            if (tid == 0) sh->target = full ? -2 : cnt;
+            consumer_barrier();
+            unsigned long long gbest = sh->red_key[0];
+#pragma unroll
+            for (int x = 1; x < NW; ++x) gbest = sh->red_key[x] < gbest ? sh->red_key[x] : gbest;
+            if (full && best_slot >= 0 && best == gbest) {
+                const unsigned long long self_key =
+                    ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
+                if (c.R > 0 || gbest < self_key) sh->target = best_slot;
+            }
+            consumer_barrier();
+
+            const int target = sh->target;
+            if (target >= 0) {
+                if (tid < LPR)
+                    *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
+                        *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
+                else if (tid < 2 * LPR)
+                    *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
+                        *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
+            }
+            if (tid == 0 && !*abort_flag) {
+                if (target >= 0) {
+                    Su[target] = a_self;
+                    posu[target] = p;
+                }
+                if (!full) c.count[u] = cnt + 1;
+                c.len[u] = p + 1;
+                evicted[u] = full ? target : -1;
+            }
+            consumer_barrier();      // w[], part[], target are reused by the next unit
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && sh->abort_flag) *status = A2SF_ERR_TIMEOUT;
+}
+
 template <typename T, int D>
 cudaError_t launch_typed(const CacheView &c, float alpha, const void *q, const void *k_new,
                          const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
@@ -232,20 +538,62 @@ cudaError_t launch_typed(const CacheView &c, float alpha, const void *q, const v
     return cudaGetLastError();
 }
 
+
+template <typename T, int D>
+cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const void *k_new,
+                          const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    const size_t smem = 128 + (size_t)kStreamStages * kChunkBytes + (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 +
+                        (size_t)kStreamConsumerWarps * D * 4 + sizeof(StreamShared);
+    if (smem > 227 * 1024) return launch_typed<T, D>(c, alpha, q, k_new, v_new, out, evicted, s);
+    auto kern = decode_step_stream_kernel<T, D>;
+    static int num_sms = 0;
+    static cudaError_t attr_err = cudaSuccess;
+    static size_t attr_smem = 0;
+    if (num_sms == 0 || smem > attr_smem) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_smem = smem;
+    }
+    if (attr_err != cudaSuccess) return attr_err;
+    int *status = decode_status_word();
+    if (!status) return cudaErrorUnknown;
+    const int grid = c.U < num_sms ? c.U : num_sms;
+    kern<<<grid, kStreamThreads, smem, s>>>(c, alpha, static_cast<const T *>(q),
+                                            static_cast<const T *>(k_new), static_cast<const T *>(v_new),
+                                            static_cast<T *>(out), evicted, status);
+    count_launch();
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
                                const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
 #define A2SF_DISPATCH(T)                                                                     \
-    (c.d == 64 ? launch_typed<T, 64>(c, alpha, q, k_new, v_new, out, evicted, s)             \
-               : launch_typed<T, 128>(c, alpha, q, k_new, v_new, out, evicted, s))
+    (c.d == 64 ? launch_stream<T, 64>(c, alpha, q, k_new, v_new, out, evicted, s)            \
+               : launch_stream<T, 128>(c, alpha, q, k_new, v_new, out, evicted, s))
     switch (c.dtype) {
     case A2SF_F32: return A2SF_DISPATCH(float);
     case A2SF_BF16: return A2SF_DISPATCH(__nv_bfloat16);
     default: return A2SF_DISPATCH(__half);
     }
 #undef A2SF_DISPATCH
+}
+
+int read_and_clear_decode_status(cudaStream_t s)
+{
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbolAsync(&v, g_decode_status, sizeof(int), 0, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return A2SF_ERR_CUDA;
+    if (v != 0 &&
+        cudaMemcpyToSymbolAsync(g_decode_status, &zero, sizeof(int), 0, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return v;
 }
 
 }  // namespace a2sf
