@@ -238,7 +238,8 @@ constexpr int kStreamConsumerWarps = 8;
 constexpr int kStreamConsumers = kStreamConsumerWarps * 32;
 constexpr int kStreamThreads = kStreamConsumers + 32;
 constexpr int kChunkBytes = 16384;
-constexpr int kStreamStages = 10;
+constexpr int kMaxStreamStages = 12;
+constexpr int kPrefetchSlots = 2;            // score/position words each consumer thread preloads
 
 __device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
 {
@@ -279,7 +280,7 @@ __device__ __forceinline__ float consumer_sum(float v, float *red)
 }
 
 struct StreamShared {
-    uint64_t full[kStreamStages], empty[kStreamStages];
+    uint64_t full[kMaxStreamStages], empty[kMaxStreamStages];
     unsigned long long red_key[kStreamConsumerWarps];
     float red[kStreamConsumerWarps];
     int target;
@@ -290,7 +291,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kStreamThreads)
 decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
                           const T *__restrict__ k_new, const T *__restrict__ v_new,
-                          T *__restrict__ out, int32_t *__restrict__ evicted, int *status)
+                          T *__restrict__ out, int32_t *__restrict__ evicted, int *status,
+                          int kStreamStages)
 {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;                    // lanes per row
@@ -365,8 +367,20 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             float *Su = c.S + (size_t)u * M;
             int32_t *posu = c.pos + (size_t)u * M;
 
+            // every global word this unit needs is requested up front, so its latency hides
+            // behind the K and V phases instead of stalling the reductions and the epilogue
             float qf[VEC];
             Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
+            const uint4 knew_raw = *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC);
+            const float vnew_val = tid < D ? Elem<T>::to_float(v_new[(size_t)u * D + tid]) : 0.f;
+            float s_pre[kPrefetchSlots];
+            int pos_pre[kPrefetchSlots];
+#pragma unroll
+            for (int x = 0; x < kPrefetchSlots; ++x) {
+                const int s_ = tid + x * kStreamConsumers;
+                s_pre[x] = s_ < cnt ? Su[s_] : 0.f;
+                pos_pre[x] = s_ < cnt ? posu[s_] : 0;
+            }
 
             // (i) logits
             for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
@@ -396,7 +410,7 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             }
             if (warp == 0) {
                 float kf[VEC];
-                Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC), kf);
+                Elem<T>::unpack(knew_raw, kf);
                 float dot = 0.f;
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
@@ -459,7 +473,7 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
                 float o = 0.f;
 #pragma unroll
                 for (int x = 0; x < NW; ++x) o += part[x * D + tid];
-                o = fmaf(e_self, Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+                o = fmaf(e_self, vnew_val, o);
                 out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
             }
 
@@ -468,11 +482,16 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             const int newest_evictable = p - c.R;
             unsigned long long best = ~0ull;
             int best_slot = -1;
-            for (int s_ = tid; s_ < cnt; s_ += kStreamConsumers) {
+            int x_pre = 0;
+            for (int s_ = tid; s_ < cnt; s_ += kStreamConsumers, ++x_pre) {
                 const float a = w[s_] / l;
-                const float sn = fmaf(alpha, Su[s_], a);
+                float s_old;
+                int ps;
+                if (x_pre == 0) { s_old = s_pre[0]; ps = pos_pre[0]; }
+                else if (x_pre == 1) { s_old = s_pre[1]; ps = pos_pre[1]; }
+                else { s_old = Su[s_]; ps = posu[s_]; }
+                const float sn = fmaf(alpha, s_old, a);
                 Su[s_] = sn;
-                const int ps = posu[s_];
                 if (full && ps <= newest_evictable) {
                     const unsigned long long key =
                         ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
@@ -543,9 +562,15 @@ template <typename T, int D>
 cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const void *k_new,
                           const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
-    const size_t smem = 128 + (size_t)kStreamStages * kChunkBytes + (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 +
-                        (size_t)kStreamConsumerWarps * D * 4 + sizeof(StreamShared);
-    if (smem > 227 * 1024) return launch_typed<T, D>(c, alpha, q, k_new, v_new, out, evicted, s);
+    const size_t fixed = 128 + (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 +
+                         (size_t)kStreamConsumerWarps * D * 4 + sizeof(StreamShared);
+    // two CTAs per SM so one CTA's reductions overlap the other's streaming; the ring takes
+    // what is left of the SM's shared memory
+    const size_t per_cta = (227 * 1024) / 2 - 1024;
+    if (fixed + 3 * kChunkBytes > per_cta) return launch_typed<T, D>(c, alpha, q, k_new, v_new, out, evicted, s);
+    int stages = (int)((per_cta - fixed) / kChunkBytes);
+    if (stages > kMaxStreamStages) stages = kMaxStreamStages;
+    const size_t smem = fixed + (size_t)stages * kChunkBytes;
     auto kern = decode_step_stream_kernel<T, D>;
     static int num_sms = 0;
     static cudaError_t attr_err = cudaSuccess;
@@ -560,10 +585,10 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     if (attr_err != cudaSuccess) return attr_err;
     int *status = decode_status_word();
     if (!status) return cudaErrorUnknown;
-    const int grid = c.U < num_sms ? c.U : num_sms;
+    const int grid = c.U < 2 * num_sms ? c.U : 2 * num_sms;
     kern<<<grid, kStreamThreads, smem, s>>>(c, alpha, static_cast<const T *>(q),
                                             static_cast<const T *>(k_new), static_cast<const T *>(v_new),
-                                            static_cast<T *>(out), evicted, status);
+                                            static_cast<T *>(out), evicted, status, stages);
     count_launch();
     return cudaGetLastError();
 }
