@@ -193,7 +193,7 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const
 // ---- cache object --------------------------------------------------------------
 
 struct CacheLayout {
-    size_t K, V, S, pos, count, len, st_q, st_k, st_v, st_out, st_ev, total;
+    size_t K, V, S, pos, count, len, sched, st_q, st_k, st_v, st_out, st_ev, total;
 };
 
 static CacheLayout cache_layout(const a2sf_params *p)
@@ -207,6 +207,7 @@ static CacheLayout cache_layout(const a2sf_params *p)
     L.pos = off; off += align_up(U * M * 4);
     L.count = off; off += align_up(U * 4);
     L.len = off; off += align_up(U * 4);
+    L.sched = off; off += align_up(2 * 4);
     L.st_q = off; off += align_up(U * d * e);
     L.st_k = off; off += align_up(U * d * e);
     L.st_v = off; off += align_up(U * d * e);
@@ -248,6 +249,7 @@ int a2sf_cache_create(const a2sf_params *p, void *device_mem, size_t bytes, a2sf
     c->view.pos = reinterpret_cast<int32_t *>(b + L.pos);
     c->view.count = reinterpret_cast<int32_t *>(b + L.count);
     c->view.len = reinterpret_cast<int32_t *>(b + L.len);
+    c->view.sched = reinterpret_cast<int32_t *>(b + L.sched);
     c->view.U = p->B * p->H; c->view.M = p->budget; c->view.R = p->recent;
     c->view.d = p->d; c->view.dtype = p->dtype; c->view.scale = eff_scale(p);
     c->st_q = b + L.st_q; c->st_k = b + L.st_k; c->st_v = b + L.st_v; c->st_out = b + L.st_out;

@@ -124,6 +124,7 @@ struct CacheView {
     float *S;             // [U][M]
     int32_t *pos;         // [U][M]
     int32_t *count, *len; // [U]
+    int32_t *sched;       // [2] unit-claim counter and finished-CTA counter of the decode kernel
     int U, M, R, d, dtype;
     float scale;
 };

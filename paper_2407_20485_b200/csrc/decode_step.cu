@@ -5,6 +5,8 @@
 //
 // Memory-bound: every K and V row of the head is read exactly once with 16-byte
 // loads, lanes laid across the row so a warp reads whole 512-byte spans.
+#include <cstdlib>
+
 #include "common.cuh"
 #include "tc_sm100.cuh"
 
@@ -255,6 +257,21 @@ __device__ __forceinline__ void consumer_barrier()
     tc::named_barrier(1, kStreamConsumers);
 }
 
+// barrier over the consumer warps that also ORs a predicate: every thread gets the same answer
+__device__ __forceinline__ bool consumer_any(bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(kStreamConsumers)
+        : "memory");
+    return r != 0;
+}
+
 __device__ __forceinline__ float consumer_max(float v, float *red)
 {
     v = warp_max(v);
@@ -279,8 +296,12 @@ __device__ __forceinline__ float consumer_sum(float v, float *red)
     return r;
 }
 
+constexpr int kUnitQueue = 4;                // units the producer may run ahead of the consumers
+
 struct StreamShared {
     uint64_t full[kMaxStreamStages], empty[kMaxStreamStages];
+    uint64_t uq_full[kUnitQueue], uq_empty[kUnitQueue];
+    int unit_q[kUnitQueue];
     unsigned long long red_key[kStreamConsumerWarps];
     float red[kStreamConsumerWarps];
     int target;
@@ -315,6 +336,7 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
 
     if (tid == 0) {
         for (int s = 0; s < kStreamStages; ++s) { tc::mbar_init(&sh->full[s], 1); tc::mbar_init(&sh->empty[s], NW); }
+        for (int x = 0; x < kUnitQueue; ++x) { tc::mbar_init(&sh->uq_full[x], 1); tc::mbar_init(&sh->uq_empty[x], NW); }
         sh->abort_flag = 0;
         tc::fence_mbar_init();
     }
@@ -333,7 +355,17 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             uint32_t g = 0;                         // chunk sequence number (same on both sides)
             uint32_t inflight_from = 0;
             bool alive = true;
-            for (int u = blockIdx.x; alive && u < c.U; u += gridDim.x) {
+            // units are claimed from a device-wide counter, so CTAs that meet cheap units or
+            // start early simply take more of them; the claim is handed to the consumers
+            // through a small queue
+            for (uint32_t n_unit = 0; alive; ++n_unit) {
+                const int qi = n_unit % kUnitQueue;
+                if (!wait(&sh->uq_empty[qi], ((n_unit / kUnitQueue) & 1) ^ 1)) { alive = false; break; }
+                int u = atomicAdd(&c.sched[0], 1);
+                if (u >= c.U) u = -1;
+                sh->unit_q[qi] = u;
+                tc::mbar_arrive(&sh->uq_full[qi]);
+                if (u < 0) break;
                 const int cnt = min(c.count[u], M);
                 for (int pass = 0; alive && pass < 2; ++pass) {
                     const uint8_t *base = static_cast<const uint8_t *>(pass == 0 ? c.K : c.V) +
@@ -359,7 +391,12 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
         // ---- consumers ---------------------------------------------------------------------
         const int sub = lane % LPR, rsel = lane / LPR;
         uint32_t g = 0;
-        for (int u = blockIdx.x; u < c.U; u += gridDim.x) {
+        for (uint32_t n_unit = 0;; ++n_unit) {
+            const int qi = n_unit % kUnitQueue;
+            const bool got = wait(&sh->uq_full[qi], (n_unit / kUnitQueue) & 1);
+            const int u = got ? sh->unit_q[qi] : -1;
+            if (consumer_any(!got) || u < 0) break;        // uniform over the consumers
+            if (lane == 0) tc::mbar_arrive(&sh->uq_empty[qi]);
             const int cnt = min(c.count[u], M);
             const int p = c.len[u];
             T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
@@ -535,7 +572,16 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
         }
     }
     __syncthreads();
-    if (tid == 0 && sh->abort_flag) *status = A2SF_ERR_TIMEOUT;
+    if (tid == 0) {
+        if (sh->abort_flag) *status = A2SF_ERR_TIMEOUT;
+        // the last CTA to leave re-arms the claim counter for the next launch
+        __threadfence();
+        if (atomicAdd(&c.sched[1], 1) == (int)gridDim.x - 1) {
+            c.sched[0] = 0;
+            c.sched[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 template <typename T, int D>
@@ -566,7 +612,8 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
                          (size_t)kStreamConsumerWarps * D * 4 + sizeof(StreamShared);
     // two CTAs per SM so one CTA's reductions overlap the other's streaming; the ring takes
     // what is left of the SM's shared memory
-    const size_t per_cta = (227 * 1024) / 2 - 1024;
+    static int ctas_per_sm = getenv("A2SF_TUNE_DECODE_CTAS") ? atoi(getenv("A2SF_TUNE_DECODE_CTAS")) : 2;
+    const size_t per_cta = (227 * 1024) / ctas_per_sm - 1024;
     if (fixed + 3 * kChunkBytes > per_cta) return launch_typed<T, D>(c, alpha, q, k_new, v_new, out, evicted, s);
     int stages = (int)((per_cta - fixed) / kChunkBytes);
     if (stages > kMaxStreamStages) stages = kMaxStreamStages;
@@ -585,7 +632,7 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     if (attr_err != cudaSuccess) return attr_err;
     int *status = decode_status_word();
     if (!status) return cudaErrorUnknown;
-    const int grid = c.U < 2 * num_sms ? c.U : 2 * num_sms;
+    const int grid = c.U < ctas_per_sm * num_sms ? c.U : ctas_per_sm * num_sms;
     kern<<<grid, kStreamThreads, smem, s>>>(c, alpha, static_cast<const T *>(q),
                                             static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                             static_cast<T *>(out), evicted, status, stages);
