@@ -302,6 +302,7 @@ struct StreamShared {
     uint64_t full[kMaxStreamStages], empty[kMaxStreamStages];
     uint64_t uq_full[kUnitQueue], uq_empty[kUnitQueue];
     int unit_q[kUnitQueue];
+    int cnt_q[kUnitQueue];
     unsigned long long red_key[kStreamConsumerWarps];
     float red[kStreamConsumerWarps];
     int target;
@@ -350,54 +351,65 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
     };
 
     if (warp == NW) {
-        // ---- producer: one lane streams K then V of every unit this CTA owns ----------------
+        // ---- producer: one lane streams K then V of every unit this CTA claims -------------
         if (lane == 0) {
-            uint32_t g = 0;                         // chunk sequence number (same on both sides)
-            uint32_t inflight_from = 0;
+            int stage = 0;
+            uint32_t phase = 0, issued = 0;
             bool alive = true;
-            // units are claimed from a device-wide counter, so CTAs that meet cheap units or
-            // start early simply take more of them; the claim is handed to the consumers
-            // through a small queue
+            // Units are claimed from a device-wide counter, so a CTA that starts early or meets
+            // short units simply takes more of them.  The claim for the NEXT unit and its row
+            // count are requested before the current unit is streamed, so neither round trip
+            // ever stalls the copy stream.
+            int u_next = atomicAdd(&c.sched[0], 1);
+            if (u_next >= c.U) u_next = -1;
+            int cnt_next = u_next >= 0 ? min(c.count[u_next], M) : 0;
             for (uint32_t n_unit = 0; alive; ++n_unit) {
+                const int u = u_next, cnt = cnt_next;
                 const int qi = n_unit % kUnitQueue;
                 if (!wait(&sh->uq_empty[qi], ((n_unit / kUnitQueue) & 1) ^ 1)) { alive = false; break; }
-                int u = atomicAdd(&c.sched[0], 1);
-                if (u >= c.U) u = -1;
                 sh->unit_q[qi] = u;
+                sh->cnt_q[qi] = cnt;
                 tc::mbar_arrive(&sh->uq_full[qi]);
                 if (u < 0) break;
-                const int cnt = min(c.count[u], M);
+                u_next = atomicAdd(&c.sched[0], 1);
+                if (u_next >= c.U) u_next = -1;
+                cnt_next = u_next >= 0 ? min(c.count[u_next], M) : 0;
                 for (int pass = 0; alive && pass < 2; ++pass) {
                     const uint8_t *base = static_cast<const uint8_t *>(pass == 0 ? c.K : c.V) +
                                           (size_t)u * M * ROWB;
-                    for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
-                        const int s = g % kStreamStages;
-                        if (!wait(&sh->empty[s], ((g / kStreamStages) & 1) ^ 1)) { alive = false; break; }
+                    for (int r0 = 0; r0 < cnt; r0 += CR) {
+                        if (!wait(&sh->empty[stage], phase ^ 1)) { alive = false; break; }
                         const uint32_t bytes = (uint32_t)min(CR, cnt - r0) * ROWB;
-                        tc::mbar_arrive_expect_tx(&sh->full[s], bytes);
-                        bulk_load(ring + s * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[s]);
+                        tc::mbar_arrive_expect_tx(&sh->full[stage], bytes);
+                        bulk_load(ring + stage * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[stage]);
+                        ++issued;
+                        if (++stage == kStreamStages) { stage = 0; phase ^= 1; }
                     }
                 }
             }
             if (!alive) {
                 // bounded chance for copies already issued to land before the CTA exits
                 int dummy = 0;
-                inflight_from = g > (uint32_t)kStreamStages ? g - kStreamStages : 0;
-                for (uint32_t x = inflight_from; x < g; ++x)
-                    tc::mbar_wait(&sh->full[x % kStreamStages], (x / kStreamStages) & 1, &dummy);
+                const uint32_t back = issued < (uint32_t)kStreamStages ? issued : (uint32_t)kStreamStages;
+                for (uint32_t x = 0; x < back; ++x) {
+                    if (stage == 0) { stage = kStreamStages; phase ^= 1; }
+                    --stage;
+                    tc::mbar_wait(&sh->full[stage], phase, &dummy);
+                }
             }
         }
     } else {
         // ---- consumers ---------------------------------------------------------------------
         const int sub = lane % LPR, rsel = lane / LPR;
-        uint32_t g = 0;
+        int stage = 0;
+        uint32_t phase = 0;
         for (uint32_t n_unit = 0;; ++n_unit) {
             const int qi = n_unit % kUnitQueue;
             const bool got = wait(&sh->uq_full[qi], (n_unit / kUnitQueue) & 1);
             const int u = got ? sh->unit_q[qi] : -1;
+            const int cnt = got ? sh->cnt_q[qi] : 0;
             if (consumer_any(!got) || u < 0) break;        // uniform over the consumers
             if (lane == 0) tc::mbar_arrive(&sh->uq_empty[qi]);
-            const int cnt = min(c.count[u], M);
             const int p = c.len[u];
             T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
             T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
@@ -420,15 +432,14 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             }
 
             // (i) logits
-            for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
-                const int s = g % kStreamStages;
-                wait(&sh->full[s], (g / kStreamStages) & 1);
-                const uint8_t *stage = ring + s * kChunkBytes;
+            for (int r0 = 0; r0 < cnt; r0 += CR) {
+                wait(&sh->full[stage], phase);
+                const uint8_t *sbase = ring + stage * kChunkBytes;
                 uint4 r[LPC];
 #pragma unroll
                 for (int x = 0; x < LPC; ++x) {
                     const int lrow = (x * NW + warp) * RPW + rsel;
-                    r[x] = *reinterpret_cast<const uint4 *>(stage + lrow * ROWB + sub * 16);
+                    r[x] = *reinterpret_cast<const uint4 *>(sbase + lrow * ROWB + sub * 16);
                 }
 #pragma unroll
                 for (int x = 0; x < LPC; ++x) {
@@ -443,7 +454,8 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
                     if (sub == 0 && row < cnt) w[row] = dot * c.scale;
                 }
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+                if (lane == 0) tc::mbar_arrive(&sh->empty[stage]);
+                if (++stage == kStreamStages) { stage = 0; phase ^= 1; }
             }
             if (warp == 0) {
                 float kf[VEC];
@@ -474,15 +486,14 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             float acc[VEC];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-            for (int r0 = 0; r0 < cnt; r0 += CR, ++g) {
-                const int s = g % kStreamStages;
-                wait(&sh->full[s], (g / kStreamStages) & 1);
-                const uint8_t *stage = ring + s * kChunkBytes;
+            for (int r0 = 0; r0 < cnt; r0 += CR) {
+                wait(&sh->full[stage], phase);
+                const uint8_t *sbase = ring + stage * kChunkBytes;
                 uint4 r[LPC];
 #pragma unroll
                 for (int x = 0; x < LPC; ++x) {
                     const int lrow = (x * NW + warp) * RPW + rsel;
-                    r[x] = *reinterpret_cast<const uint4 *>(stage + lrow * ROWB + sub * 16);
+                    r[x] = *reinterpret_cast<const uint4 *>(sbase + lrow * ROWB + sub * 16);
                 }
 #pragma unroll
                 for (int x = 0; x < LPC; ++x) {
@@ -496,7 +507,8 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
                     }
                 }
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(&sh->empty[s]);
+                if (lane == 0) tc::mbar_arrive(&sh->empty[stage]);
+                if (++stage == kStreamStages) { stage = 0; phase ^= 1; }
             }
 #pragma unroll
             for (int o = LPR; o < 32; o <<= 1)
