@@ -85,9 +85,11 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
     uint8_t *Qs = smem + kTileBytes;
     ScoreShared *sh = reinterpret_cast<ScoreShared *>(smem + kTileBytes * (1 + kScoreStages));
 
-    const int u = blockIdx.x, kb = blockIdx.y;
-    const int b = u / a.H, h = u % a.H;
+    // CTAs of one unit are adjacent in the grid, so they run together and share the unit's
+    // Q and K tiles through L2
     const int ntile_total = (a.n + kBlk - 1) / kBlk;
+    const int u = blockIdx.x / ntile_total, kb = blockIdx.x % ntile_total;
+    const int b = u / a.H, h = u % a.H;
     const int ntiles = ntile_total - kb;               // query-row tiles kb .. last
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sh->abort_flag;
@@ -288,9 +290,11 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     // split into two bf16 terms (p = hi + lo, |lo| <= 2^-9 |hi|) and both are multiplied
     // with V.  fp16 keeps 11 bits and needs no second term.
     constexpr bool kSplitP = std::is_same<T, __nv_bfloat16>::value;
-    const int u = blockIdx.x;
+    // CTAs of one unit are adjacent in the grid (longest rows first), so they run together
+    // and share the unit's K and V tiles through L2
     const int T_total = (a.n + kBlk - 1) / kBlk;
-    const int rb = T_total - 1 - blockIdx.y;            // longest rows first
+    const int u = blockIdx.x / T_total;
+    const int rb = T_total - 1 - blockIdx.x % T_total;
     const int nt = rb + 1;                              // key tiles 0 .. rb
     const int b = u / a.H, h = u % a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -572,7 +576,7 @@ bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillA
 bool prefill_tc_supported(int dtype, const PrefillArgs &a)
 {
     return (dtype == A2SF_BF16 || dtype == A2SF_F16) && a.d == kD &&
-           (a.n + kBlk - 1) / kBlk <= 65535;
+           (size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk) < 0x7fffffffull;
 }
 
 cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
@@ -596,7 +600,7 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
     aa.n = a.n; aa.H = a.H;
     aa.sl2 = a.scale * kLog2e;
-    dim3 grid(a.B * a.H, (a.n + kBlk - 1) / kBlk);
+    const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
     if (dtype == A2SF_BF16)
         attn_pass_tc<__nv_bfloat16><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
     else
@@ -621,7 +625,7 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     sa.lse = a.lse; sa.scores = a.scores; sa.n = a.n; sa.H = a.H;
     sa.sl2 = a.scale * kLog2e;
     sa.neg_log2_alpha = a.alpha > 0.f ? -log2f(a.alpha) : INFINITY;
-    dim3 grid(a.B * a.H, (a.n + kBlk - 1) / kBlk);
+    const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
     score_pass_tc<<<grid, kScoreThreads, kScoreSmemBytes, s>>>(mq, mk, sa, dtype == A2SF_BF16 ? 1 : 0);
     count_launch();
     return cudaGetLastError();
