@@ -409,7 +409,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
         const int i = rb * kBlk + r;
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-        float m_used = -INFINITY, l = 0.f;
+        float m_used = 0.f, l = 0.f;
         bool ok = true;
         for (int t = 0; ok && t < nt; ++t) {
             const int sb = t & 1;
@@ -417,85 +417,82 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             tc_fence_after_sync();
             const uint32_t s_addr = tmem_base + sb * kBlk + lane_off;
             const bool diag = (t == nt - 1);
-            // pass A: row maximum of the scaled logits (log2 domain)
-            float tmax = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < kBlk / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_wait_ld();
+            // the whole logits row comes into registers with one wait; the buffer is free again
+            uint32_t v[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v[c]);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            mbar_arrive(&sh->s_empty[sb]);
+            // exponent arguments relative to the current reference maximum (log2 domain)
+            float xmax = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int x = 0; x < 32; ++x) {
-                    float sv = __uint_as_float(v[x]) * a.sl2;
-                    if (diag && c * 32 + x > r) sv = -INFINITY;        // causal mask
-                    tmax = fmaxf(tmax, sv);
+                    float e = fmaf(__uint_as_float(v[c][x]), a.sl2, -m_used);
+                    if (diag && c * 32 + x > r) e = -INFINITY;            // causal mask
+                    xmax = fmaxf(xmax, e);
+                    v[c][x] = __float_as_uint(e);
                 }
-            }
-            // lazy maximum: keep the old reference unless the new maximum exceeds it by 2^8
+            // Lazy maximum: the reference moves only on the first tile or when the row maximum
+            // exceeds it by more than 2^8; otherwise probabilities up to 256 are simply kept.
             float factor = 1.f;
-            bool grow = false;
-            if (t == 0) {
-                m_used = tmax;
-            } else if (tmax > m_used + kRescaleThreshold) {
-                factor = ex2_approx(m_used - tmax);
-                m_used = tmax;
-                grow = true;
+            const bool grow = (t == 0) || (xmax > kRescaleThreshold);
+            if (grow) {
+                m_used += xmax;
+                factor = t == 0 ? 0.f : ex2_approx(-xmax);
             }
+            const float shift = grow ? xmax : 0.f;
+            float rowsum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    const float pv = ex2_approx(__uint_as_float(v[c][x]) - shift);   // masked -> 0
+                    rowsum += pv;
+                    v[c][x] = __float_as_uint(pv);
+                }
+            l = fmaf(l, factor, rowsum);
             // P(t-1) has been consumed and O holds tiles 0..t-1 once p_empty completes
             if (t > 0 && !mbar_wait(&sh->p_empty, (t - 1) & 1, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            if (__any_sync(0xffffffffu, grow)) {
-                l *= factor;
+            if (t > 0 && __any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
                 for (int c = 0; c < kD / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem_o + lane_off + c * 32, v);
+                    uint32_t o[32];
+                    tmem_ld32(tmem_o + lane_off + c * 32, o);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) v[x] = __float_as_uint(__uint_as_float(v[x]) * factor);
-                    tmem_st32(tmem_o + lane_off + c * 32, v);
+                    for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * factor);
+                    tmem_st32(tmem_o + lane_off + c * 32, o);
                 }
                 tmem_wait_st();
             }
-            // pass B: probabilities, row sum (unrounded), P tile to shared memory
-            float rowsum = 0.f;
-            const float neg_m = -m_used;
-#pragma unroll 1
-            for (int c = 0; c < kBlk / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(s_addr + c * 32, v);
-                tmem_wait_ld();
-                uint32_t pk[16], pl[16];
+            // P tile (rounded to the storage type; for bf16 also the rounding remainder) to
+            // shared memory in the swizzled K-major layout
 #pragma unroll
-                for (int x = 0; x < 32; x += 2) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(v[x]), a.sl2, neg_m));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(v[x + 1]), a.sl2, neg_m));
-                    if (diag) {
-                        if (c * 32 + x > r) p0 = 0.f;
-                        if (c * 32 + x + 1 > r) p1 = 0.f;
-                    }
-                    rowsum += p0 + p1;
-                    const uint32_t hi = pack2<T>(p0, p1);
-                    pk[x >> 1] = hi;
-                    if (kSplitP)      // a bf16 is the upper half of an fp32
-                        pl[x >> 1] = pack2<T>(p0 - __uint_as_float(hi << 16),
-                                              p1 - __uint_as_float(hi & 0xffff0000u));
-                }
-                // columns c*32 .. c*32+31 = 16-byte chunks (c&1)*4 .. +3 of half c>>1
+            for (int c = 0; c < 4; ++c) {
                 const int row_off = (c >> 1) * kHalfBytes + r * 128;
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
+                    uint32_t hi[4], lo[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float p0 = __uint_as_float(v[c][q4 * 8 + 2 * e]);
+                        const float p1 = __uint_as_float(v[c][q4 * 8 + 2 * e + 1]);
+                        hi[e] = pack2<T>(p0, p1);
+                        if (kSplitP)      // a bf16 is the upper half of an fp32
+                            lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
+                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    }
                     const int chunk = ((c & 1) * 4 + q4) ^ (r & 7);
-                    *reinterpret_cast<uint4 *>(Ps + row_off + chunk * 16) =
-                        make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+                    *reinterpret_cast<uint4 *>(Ps + row_off + chunk * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
                     if (kSplitP)
-                        *reinterpret_cast<uint4 *>(Pl + row_off + chunk * 16) =
-                            make_uint4(pl[q4 * 4], pl[q4 * 4 + 1], pl[q4 * 4 + 2], pl[q4 * 4 + 3]);
+                        *reinterpret_cast<uint4 *>(Pl + row_off + chunk * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
                 }
             }
-            l += rowsum;
             tc_fence_before_sync();
-            mbar_arrive(&sh->s_empty[sb]);            // the logits buffer may be overwritten
             fence_async_smem();                       // P stores -> visible to the tensor core
             mbar_arrive(&sh->p_full);
         }
