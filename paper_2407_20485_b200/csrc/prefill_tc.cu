@@ -223,14 +223,16 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //                         current tile is in the softmax warps)
 //   softmax warps      : one thread per row; running maximum kept lazily (the accumulator is
 //                         rescaled only when the maximum grows by more than 2^8), P rounded to
-//                         the storage type and written to shared memory in the 128-byte-swizzled
-//                         K-major layout the MMA reads; the row sum uses the unrounded values
+//                         the storage type and written back to TENSOR memory, from where the MMA
+//                         reads it as its A operand (shared-memory bandwidth is the scarce
+//                         resource: operands read from it at 128x128x16 per instruction already
+//                         saturate it); the row sum uses the unrounded values
 //   O += P V           -> TMEM; V is consumed as an MN-major operand straight from its TMA tile
 // Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
 // softmax + epilogue.
 // ============================================================================================
 constexpr int kAttnThreads = 192;
-constexpr int kKvStages = 2;
+constexpr int kKvStages = 3;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
 
 struct AttnArgs {
@@ -248,8 +250,8 @@ struct AttnShared {
     int abort_flag;
 };
 
-// Q, P (high part), P (low part, bf16 only), K ring, V ring
-constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (3 + 2 * kKvStages) + sizeof(AttnShared);
+// Q, K ring, V ring
+constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (1 + 2 * kKvStages) + sizeof(AttnShared);
 
 template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
 template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b)
@@ -278,9 +280,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                 ~uintptr_t(1023));
     uint8_t *Qs = smem;
-    uint8_t *Ps = smem + kTileBytes;
-    uint8_t *Pl = smem + 2 * kTileBytes;
-    uint8_t *Ks = smem + 3 * kTileBytes;
+    uint8_t *Ks = smem + kTileBytes;
     uint8_t *Vs = Ks + kKvStages * kTileBytes;
     AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kKvStages * kTileBytes);
 
@@ -320,7 +320,10 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
-    const uint32_t tmem_o = tmem_base + 2 * kBlk;        // S0 | S1 | O
+    // tensor memory columns: S0 | S1 | O | P (high) | P (low)
+    const uint32_t tmem_o = tmem_base + 2 * kBlk;
+    const uint32_t tmem_ph = tmem_base + 3 * kBlk;
+    const uint32_t tmem_pl = tmem_ph + kBlk / 2;
 
     if (warp == 0) {
         // ---- TMA producer -------------------------------------------------------------
@@ -360,7 +363,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
             const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
-            const uint32_t q_addr = smem_u32(Qs), p_addr = smem_u32(Ps), pl_addr = smem_u32(Pl);
+            const uint32_t q_addr = smem_u32(Qs);
             auto issue_s = [&](int t) -> bool {
                 const int s = t % kKvStages;
                 const int sb = t & 1;
@@ -383,20 +386,16 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 const uint32_t v_addr = smem_u32(Vs + s * kTileBytes);
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k) {
-                    // A = P: 16 keys = 32 bytes along the swizzled row; B = V: 16 keys = two
-                    // 8-row groups of 1024 bytes, the two 64-wide d halves 16 KB apart
-                    const uint64_t adesc =
-                        make_sdesc_sw128(p_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
+                    // A = P from tensor memory: 16 keys = 8 columns; B = V: 16 keys = two 8-row
+                    // groups of 1024 bytes, the two 64-wide d halves 16 KB apart
                     const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                    umma_ss(tmem_o, adesc, bdesc, idesc_pv, (t > 0) || (k > 0));
+                    umma_ts(tmem_o, tmem_ph + k * 8, bdesc, idesc_pv, (t > 0) || (k > 0));
                 }
                 if (kSplitP) {
 #pragma unroll
                     for (int k = 0; k < kBlk / 16; ++k) {
-                        const uint64_t adesc =
-                            make_sdesc_sw128(pl_addr + (k >> 2) * kHalfBytes + (k & 3) * 32, 16, 1024);
                         const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                        umma_ss(tmem_o, adesc, bdesc, idesc_pv, 1);
+                        umma_ts(tmem_o, tmem_pl + k * 8, bdesc, idesc_pv, 1);
                     }
                 }
                 umma_commit(&sh->v_empty[s]);
@@ -470,30 +469,24 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 tmem_wait_st();
             }
             // P tile (rounded to the storage type; for bf16 also the rounding remainder) to
-            // shared memory in the swizzled K-major layout
+            // tensor memory: two 16-bit values per 32-bit column, 32 keys = 16 columns
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                const int row_off = (c >> 1) * kHalfBytes + r * 128;
+                uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint32_t hi[4], lo[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const float p0 = __uint_as_float(v[c][q4 * 8 + 2 * e]);
-                        const float p1 = __uint_as_float(v[c][q4 * 8 + 2 * e + 1]);
-                        hi[e] = pack2<T>(p0, p1);
-                        if (kSplitP)      // a bf16 is the upper half of an fp32
-                            lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
-                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
-                    }
-                    const int chunk = ((c & 1) * 4 + q4) ^ (r & 7);
-                    *reinterpret_cast<uint4 *>(Ps + row_off + chunk * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-                    if (kSplitP)
-                        *reinterpret_cast<uint4 *>(Pl + row_off + chunk * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = __uint_as_float(v[c][2 * e]);
+                    const float p1 = __uint_as_float(v[c][2 * e + 1]);
+                    hi[e] = pack2<T>(p0, p1);
+                    if (kSplitP)      // a bf16 is the upper half of an fp32
+                        lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
+                                         p1 - __uint_as_float(hi[e] & 0xffff0000u));
                 }
+                tmem_st16(tmem_ph + lane_off + c * 16, hi);
+                if (kSplitP) tmem_st16(tmem_pl + lane_off + c * 16, lo);
             }
+            tmem_wait_st();
             tc_fence_before_sync();
-            fence_async_smem();                       // P stores -> visible to the tensor core
             mbar_arrive(&sh->p_full);
         }
         // ---- epilogue ---------------------------------------------------------------------
