@@ -228,10 +228,14 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //                         resource: operands read from it at 128x128x16 per instruction already
 //                         saturate it); the row sum uses the unrounded values
 //   O += P V           -> TMEM; V is consumed as an MN-major operand straight from its TMA tile
-// Warp roles (192 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
-// softmax + epilogue.
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-9
+// softmax + epilogue.  A row is shared by two threads (one per 64-column half): a single
+// warp per scheduler cannot issue the softmax arithmetic fast enough to keep up with the
+// tensor core, two interleaved warps can.  The halves exchange their row maxima through
+// shared memory once per tile and their row sums once at the end.
 // ============================================================================================
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 320;            // producer warp, MMA warp, 8 softmax warps
+constexpr int kSoftmaxThreads = 256;
 constexpr int kKvStages = 3;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
 
@@ -248,6 +252,8 @@ struct AttnShared {
     uint64_t s_full[2], s_empty[2], p_full, p_empty;
     uint32_t tmem_base;
     int abort_flag;
+    float xmax[2][2][kBlk];     // [tile parity][column half][row]
+    float lsum[2][kBlk];        // [column half][row]
 };
 
 // Q, K ring, V ring
@@ -306,8 +312,8 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             mbar_init(&sh->k_full[s], 1); mbar_init(&sh->k_empty[s], 1);
             mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1);
         }
-        for (int x = 0; x < 2; ++x) { mbar_init(&sh->s_full[x], 1); mbar_init(&sh->s_empty[x], kBlk); }
-        mbar_init(&sh->p_full, kBlk);
+        for (int x = 0; x < 2; ++x) { mbar_init(&sh->s_full[x], 1); mbar_init(&sh->s_empty[x], kSoftmaxThreads); }
+        mbar_init(&sh->p_full, kSoftmaxThreads);
         mbar_init(&sh->p_empty, 1);
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -403,37 +409,47 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             }
         }
     } else {
-        // ---- softmax + epilogue: one thread per query row ------------------------------
-        const int quarter = warp & 3;
+        // ---- softmax + epilogue: two threads per query row (64 columns each) ---------------
+        const int quarter = warp & 3;                      // TMEM lanes this warp may touch
+        const int hsel = (warp - 2) >> 2;                  // column half
         const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
         const int i = rb * kBlk + r;
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+        const int col0 = hsel * 64;
+        // A failed wait poisons the CTA: later waits return at once, the loop keeps its shape
+        // (so every thread still meets the named barrier) and the status word reports it.
+        auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
+            if (*abort_flag) return false;
+            return mbar_wait(bar, parity, abort_flag);
+        };
         float m_used = 0.f, l = 0.f;
-        bool ok = true;
-        for (int t = 0; ok && t < nt; ++t) {
+        for (int t = 0; t < nt; ++t) {
             const int sb = t & 1;
-            if (!mbar_wait(&sh->s_full[sb], (t >> 1) & 1, abort_flag)) { ok = false; break; }
+            wait(&sh->s_full[sb], (t >> 1) & 1);
             tc_fence_after_sync();
-            const uint32_t s_addr = tmem_base + sb * kBlk + lane_off;
+            const uint32_t s_addr = tmem_base + sb * kBlk + lane_off + col0;
             const bool diag = (t == nt - 1);
-            // the whole logits row comes into registers with one wait; the buffer is free again
-            uint32_t v[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, v[c]);
+            // this thread's half of the logits row comes into registers with one wait
+            uint32_t v[2][32];
+            tmem_ld32(s_addr, v[0]);
+            tmem_ld32(s_addr + 32, v[1]);
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(&sh->s_empty[sb]);
             // exponent arguments relative to the current reference maximum (log2 domain)
             float xmax = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
                 for (int x = 0; x < 32; ++x) {
                     float e = fmaf(__uint_as_float(v[c][x]), a.sl2, -m_used);
-                    if (diag && c * 32 + x > r) e = -INFINITY;            // causal mask
+                    if (diag && col0 + c * 32 + x > r) e = -INFINITY;     // causal mask
                     xmax = fmaxf(xmax, e);
                     v[c][x] = __float_as_uint(e);
                 }
+            sh->xmax[t & 1][hsel][r] = xmax;
+            named_barrier(1, kSoftmaxThreads);
+            xmax = fmaxf(xmax, sh->xmax[t & 1][hsel ^ 1][r]);
             // Lazy maximum: the reference moves only on the first tile or when the row maximum
             // exceeds it by more than 2^8; otherwise probabilities up to 256 are simply kept.
             float factor = 1.f;
@@ -442,36 +458,47 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 m_used += xmax;
                 factor = t == 0 ? 0.f : ex2_approx(-xmax);
             }
-            const float shift = grow ? xmax : 0.f;
             float rowsum = 0.f;
+            if (__any_sync(0xffffffffu, grow)) {
+                const float shift = grow ? xmax : 0.f;
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    const float pv = ex2_approx(__uint_as_float(v[c][x]) - shift);   // masked -> 0
-                    rowsum += pv;
-                    v[c][x] = __float_as_uint(pv);
-                }
+                    for (int x = 0; x < 32; ++x) {
+                        const float pv = ex2_approx(__uint_as_float(v[c][x]) - shift);   // masked -> 0
+                        rowsum += pv;
+                        v[c][x] = __float_as_uint(pv);
+                    }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 2; ++c)
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) {
+                        const float pv = ex2_approx(__uint_as_float(v[c][x]));
+                        rowsum += pv;
+                        v[c][x] = __float_as_uint(pv);
+                    }
+            }
             l = fmaf(l, factor, rowsum);
             // P(t-1) has been consumed and O holds tiles 0..t-1 once p_empty completes
-            if (t > 0 && !mbar_wait(&sh->p_empty, (t - 1) & 1, abort_flag)) { ok = false; break; }
+            if (t > 0) wait(&sh->p_empty, (t - 1) & 1);
             tc_fence_after_sync();
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
 #pragma unroll 1
-                for (int c = 0; c < kD / 32; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t o[32];
-                    tmem_ld32(tmem_o + lane_off + c * 32, o);
+                    tmem_ld32(tmem_o + lane_off + col0 + c * 32, o);
                     tmem_wait_ld();
 #pragma unroll
                     for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * factor);
-                    tmem_st32(tmem_o + lane_off + c * 32, o);
+                    tmem_st32(tmem_o + lane_off + col0 + c * 32, o);
                 }
                 tmem_wait_st();
             }
-            // P tile (rounded to the storage type; for bf16 also the rounding remainder) to
-            // tensor memory: two 16-bit values per 32-bit column, 32 keys = 16 columns
+            // P (rounded to the storage type; for bf16 also the rounding remainder) to tensor
+            // memory: two 16-bit values per 32-bit column, 32 keys = 16 columns
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t hi[16], lo[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
@@ -482,22 +509,26 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                         lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
                                          p1 - __uint_as_float(hi[e] & 0xffff0000u));
                 }
-                tmem_st16(tmem_ph + lane_off + c * 16, hi);
-                if (kSplitP) tmem_st16(tmem_pl + lane_off + c * 16, lo);
+                tmem_st16(tmem_ph + lane_off + (hsel * 2 + c) * 16, hi);
+                if (kSplitP) tmem_st16(tmem_pl + lane_off + (hsel * 2 + c) * 16, lo);
             }
             tmem_wait_st();
             tc_fence_before_sync();
             mbar_arrive(&sh->p_full);
         }
         // ---- epilogue ---------------------------------------------------------------------
-        if (ok && mbar_wait(&sh->p_empty, (nt - 1) & 1, abort_flag)) {
-            tc_fence_after_sync();
+        sh->lsum[hsel][r] = l;
+        named_barrier(1, kSoftmaxThreads);
+        l += sh->lsum[hsel ^ 1][r];
+        const bool done = wait(&sh->p_empty, (nt - 1) & 1);
+        tc_fence_after_sync();
+        if (done) {
             const float inv = 1.f / l;
-            T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t;
+            T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t + col0;
 #pragma unroll 1
-            for (int c = 0; c < kD / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tmem_o + lane_off + c * 32, v);
+            for (int c = 0; c < 2; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem_o + lane_off + col0 + c * 32, o);
                 tmem_wait_ld();
                 if (i < a.n) {
 #pragma unroll
@@ -505,13 +536,13 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                         uint32_t w[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            w[e] = pack2<T>(__uint_as_float(v[q4 * 8 + 2 * e]) * inv,
-                                            __uint_as_float(v[q4 * 8 + 2 * e + 1]) * inv);
+                            w[e] = pack2<T>(__uint_as_float(o[q4 * 8 + 2 * e]) * inv,
+                                            __uint_as_float(o[q4 * 8 + 2 * e + 1]) * inv);
                         *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
             }
-            if (i < a.n) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
+            if (i < a.n && hsel == 0) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
         }
     }
 
