@@ -236,7 +236,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 // ============================================================================================
 constexpr int kAttnThreads = 320;            // producer warp, MMA warp, 8 softmax warps
 constexpr int kSoftmaxThreads = 256;
-constexpr int kKvStages = 3;
+constexpr int kKStages = 3;                  // K tiles in flight
+constexpr int kVStages = 2;                  // V tiles in flight
 constexpr float kRescaleThreshold = 8.0f;     // log2 units
 
 struct AttnArgs {
@@ -248,7 +249,7 @@ struct AttnArgs {
 };
 
 struct AttnShared {
-    uint64_t q_full, k_full[kKvStages], k_empty[kKvStages], v_full[kKvStages], v_empty[kKvStages];
+    uint64_t q_full, k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
     uint64_t s_full[2], s_empty[2], p_full, p_empty;
     uint32_t tmem_base;
     int abort_flag;
@@ -257,7 +258,8 @@ struct AttnShared {
 };
 
 // Q, K ring, V ring
-constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (1 + 2 * kKvStages) + sizeof(AttnShared);
+constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (1 + kKStages + kVStages) + sizeof(AttnShared);
+static_assert(kAttnSmemBytes <= 227 * 1024, "attention pass shared memory");
 
 template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
 template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b)
@@ -287,8 +289,8 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                                                 ~uintptr_t(1023));
     uint8_t *Qs = smem;
     uint8_t *Ks = smem + kTileBytes;
-    uint8_t *Vs = Ks + kKvStages * kTileBytes;
-    AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kKvStages * kTileBytes);
+    uint8_t *Vs = Ks + kKStages * kTileBytes;
+    AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kVStages * kTileBytes);
 
     constexpr int ab_fmt = std::is_same<T, __nv_bfloat16>::value ? 1 : 0;
     // A bf16 probability keeps 8 significand bits; where the products p*v cancel, that
@@ -308,10 +310,8 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
 
     if (threadIdx.x == 0) {
         mbar_init(&sh->q_full, 1);
-        for (int s = 0; s < kKvStages; ++s) {
-            mbar_init(&sh->k_full[s], 1); mbar_init(&sh->k_empty[s], 1);
-            mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1);
-        }
+        for (int s = 0; s < kKStages; ++s) { mbar_init(&sh->k_full[s], 1); mbar_init(&sh->k_empty[s], 1); }
+        for (int s = 0; s < kVStages; ++s) { mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1); }
         for (int x = 0; x < 2; ++x) { mbar_init(&sh->s_full[x], 1); mbar_init(&sh->s_empty[x], kSoftmaxThreads); }
         mbar_init(&sh->p_full, kSoftmaxThreads);
         mbar_init(&sh->p_empty, 1);
@@ -340,16 +340,15 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rb * kBlk, h, b);
             int issued = 0;
             for (int t = 0; t < nt; ++t) {
-                const int s = t % kKvStages;
-                const uint32_t ph = (t / kKvStages) & 1;
-                if (!mbar_wait(&sh->k_empty[s], ph ^ 1, abort_flag)) break;
-                mbar_arrive_expect_tx(&sh->k_full[s], kTileBytes);
-                tma_load_4d(Ks + s * kTileBytes, &tmap_k, &sh->k_full[s], 0, t * kBlk, h, b);
-                tma_load_4d(Ks + s * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[s], 64, t * kBlk, h, b);
-                if (!mbar_wait(&sh->v_empty[s], ph ^ 1, abort_flag)) { issued = -(t + 1); break; }
-                mbar_arrive_expect_tx(&sh->v_full[s], kTileBytes);
-                tma_load_4d(Vs + s * kTileBytes, &tmap_v, &sh->v_full[s], 0, t * kBlk, h, b);
-                tma_load_4d(Vs + s * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[s], 64, t * kBlk, h, b);
+                const int ks = t % kKStages, vs = t % kVStages;
+                if (!mbar_wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1, abort_flag)) break;
+                mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
+                tma_load_4d(Ks + ks * kTileBytes, &tmap_k, &sh->k_full[ks], 0, t * kBlk, h, b);
+                tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[ks], 64, t * kBlk, h, b);
+                if (!mbar_wait(&sh->v_empty[vs], ((t / kVStages) & 1) ^ 1, abort_flag)) { issued = -(t + 1); break; }
+                mbar_arrive_expect_tx(&sh->v_full[vs], kTileBytes);
+                tma_load_4d(Vs + vs * kTileBytes, &tmap_v, &sh->v_full[vs], 0, t * kBlk, h, b);
+                tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[vs], 64, t * kBlk, h, b);
                 issued = t + 1;
             }
             if (*abort_flag) {
@@ -357,10 +356,10 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 int dummy = 0;
                 const int kdone = issued < 0 ? -issued : issued;
                 const int vdone = issued < 0 ? -issued - 1 : issued;
-                for (int t = max(0, kdone - kKvStages); t < kdone; ++t)
-                    mbar_wait(&sh->k_full[t % kKvStages], (t / kKvStages) & 1, &dummy);
-                for (int t = max(0, vdone - kKvStages); t < vdone; ++t)
-                    mbar_wait(&sh->v_full[t % kKvStages], (t / kKvStages) & 1, &dummy);
+                for (int t = max(0, kdone - kKStages); t < kdone; ++t)
+                    mbar_wait(&sh->k_full[t % kKStages], (t / kKStages) & 1, &dummy);
+                for (int t = max(0, vdone - kVStages); t < vdone; ++t)
+                    mbar_wait(&sh->v_full[t % kVStages], (t / kVStages) & 1, &dummy);
                 mbar_wait(&sh->q_full, 0, &dummy);
             }
         }
@@ -371,9 +370,9 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
             const uint32_t q_addr = smem_u32(Qs);
             auto issue_s = [&](int t) -> bool {
-                const int s = t % kKvStages;
+                const int s = t % kKStages;
                 const int sb = t & 1;
-                if (!mbar_wait(&sh->k_full[s], (t / kKvStages) & 1, abort_flag)) return false;
+                if (!mbar_wait(&sh->k_full[s], (t / kKStages) & 1, abort_flag)) return false;
                 if (!mbar_wait(&sh->s_empty[sb], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
                 tc_fence_after_sync();
                 issue_qk_mma(tmem_base + sb * kBlk, q_addr, smem_u32(Ks + s * kTileBytes), idesc_qk);
@@ -385,9 +384,9 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             ok = ok && issue_s(0);
             for (int t = 0; ok && t < nt; ++t) {
                 if (t + 1 < nt && !issue_s(t + 1)) break;
-                const int s = t % kKvStages;
+                const int s = t % kVStages;
                 if (!mbar_wait(&sh->p_full, t & 1, abort_flag)) break;
-                if (!mbar_wait(&sh->v_full[s], (t / kKvStages) & 1, abort_flag)) break;
+                if (!mbar_wait(&sh->v_full[s], (t / kVStages) & 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t v_addr = smem_u32(Vs + s * kTileBytes);
 #pragma unroll
