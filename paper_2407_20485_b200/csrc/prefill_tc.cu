@@ -68,7 +68,7 @@ __device__ __forceinline__ void issue_qk_mma(uint32_t d_tmem, uint32_t a_addr, u
     }
 }
 
-__global__ void __launch_bounds__(kScoreThreads)
+__global__ void __launch_bounds__(kScoreThreads, 2)
 score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
               ScoreArgs a, int ab_fmt)
 {
@@ -168,39 +168,47 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         const int et = threadIdx.x - 64;            // 0..127
         const float *lse = a.lse + (size_t)u * a.n;
         float sum = 0.f;
+        // row constant c_i = lse_i*log2e + (n-1-i)*(-log2 alpha); rows past n give +inf.
+        // The value for the NEXT tile is requested one tile ahead so its global-memory latency
+        // never sits between two tiles.
+        auto row_const = [&](int i) -> float {
+            if (i >= a.n) return INFINITY;
+            const int age = a.n - 1 - i;
+            return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * a.neg_log2_alpha);
+        };
+        float c_next = row_const(kb * kBlk + et);
         for (int it = 0; it < ntiles; ++it) {
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int i0 = (kb + it) * kBlk;
-            {   // row constants c_i = lse_i*log2e + (n-1-i)*(-log2 alpha); rows past n give +inf
-                const int i = i0 + et;
-                float cv = INFINITY;
-                if (i < a.n) {
-                    const int age = a.n - 1 - i;
-                    cv = fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * a.neg_log2_alpha);
-                }
-                sh->cbuf[it & 1][et] = cv;
-            }
+            sh->cbuf[it & 1][et] = c_next;
             mbar_arrive(&sh->c_full[acc]);       // release: the row constants are published
+            if (it + 1 < ntiles) c_next = row_const(i0 + kBlk + et);
             if (!mbar_wait(&sh->c_full[acc], aph, abort_flag)) break;
             if (!mbar_wait(&sh->acc_full[acc], aph, abort_flag)) break;
             tc_fence_after_sync();
             const float *cb = sh->cbuf[it & 1];
             const bool diag = (it == 0);
-#pragma unroll 1
-            for (int c = 0; c < kBlk / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tmem_base + acc * kBlk + c * 32 + ((uint32_t)(quarter * 32) << 16), r);
-                tmem_wait_ld();
+            // the whole 128-row strip of this key comes into registers with one wait, and the
+            // accumulator buffer goes back to the tensor core before the arithmetic starts
+            uint32_t r[4][32];
+            const uint32_t t_addr = tmem_base + acc * kBlk + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    float pw = ex2_approx(fmaf(__uint_as_float(r[x]), a.sl2, -cb[c * 32 + x]));
-                    if (diag) pw = (i0 + c * 32 + x >= j) ? pw : 0.f;    // causal: rows i >= j
-                    sum += pw;
-                }
-            }
+            for (int c = 0; c < 4; ++c) tmem_ld32(t_addr + c * 32, r[c]);
+            tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(&sh->acc_empty[acc]);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float part = 0.f;
+#pragma unroll
+                for (int x = 0; x < 32; ++x) {
+                    float pw = ex2_approx(fmaf(__uint_as_float(r[c][x]), a.sl2, -cb[c * 32 + x]));
+                    if (diag) pw = (i0 + c * 32 + x >= j) ? pw : 0.f;    // causal: rows i >= j
+                    part += pw;
+                }
+                sum += part;
+            }
         }
         if (j < a.n && !*abort_flag) a.scores[(size_t)u * a.n + j] = sum;
     }
