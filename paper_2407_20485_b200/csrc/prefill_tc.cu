@@ -2,12 +2,14 @@
 //
 //   score pass (paper Eq. 5-6):  S_j = sum_{i>=j} alpha^(n-1-i) * exp(s_ij - lse_i)
 //     One CTA owns 128 keys.  The logits are recomputed transposed, S^T = K_blk * Q_tile^T,
-//     so that a key is a TMEM lane: the thread that owns the lane sums its key's
-//     probabilities over all query rows i >= j in ascending order.  No cross-thread
-//     reduction and no atomics: the result is deterministic.
+//     so that a key is a TMEM lane: the threads that own the lane sum its key's
+//     probabilities over all query rows i >= j in a fixed order.  No atomics: the result
+//     is deterministic.
 //
-// Warp roles per CTA (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and
-// TMEM owner, warps 2-5 = epilogue (one TMEM lane quarter each).
+// Warp roles per CTA (320 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 2-9 = epilogue.  A key is shared by two threads, one per 64-row half of the
+// query tile (more warps per scheduler keep the special-function unit fed); each keeps its
+// own running sum in row order and the two are added once at the end, in a fixed order.
 #include <mutex>
 #include <type_traits>
 
@@ -28,7 +30,8 @@ constexpr int kD = 128;
 constexpr int kHalfBytes = kBlk * 64 * 2;   // one 64-column swizzled half of a tile: 16 KB
 constexpr int kTileBytes = 2 * kHalfBytes;  // 32 KB
 constexpr int kScoreStages = 2;
-constexpr int kScoreThreads = 192;
+constexpr int kScoreThreads = 320;           // producer warp, MMA warp, 8 epilogue warps
+constexpr int kScoreEpiThreads = 256;
 
 struct ScoreArgs {
     const float *lse;     // [U][n]
@@ -43,6 +46,7 @@ struct ScoreShared {
     uint32_t tmem_base;
     int abort_flag;
     float cbuf[2][kBlk];
+    float part[kBlk];           // upper-half partial sums, added to the lower half at the end
 };
 
 constexpr size_t kScoreSmemBytes = 1024 /*alignment slack*/ + kTileBytes * (1 + kScoreStages) +
@@ -99,8 +103,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         for (int s = 0; s < kScoreStages; ++s) { mbar_init(&sh->q_full[s], 1); mbar_init(&sh->q_empty[s], 1); }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sh->acc_full[x], 1);
-            mbar_init(&sh->acc_empty[x], kBlk);
-            mbar_init(&sh->c_full[x], kBlk);
+            mbar_init(&sh->acc_empty[x], kScoreEpiThreads);
+            mbar_init(&sh->c_full[x], kScoreEpiThreads);
         }
         sh->abort_flag = 0;
         fence_mbar_init();
@@ -161,56 +165,72 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             }
         }
     } else {
-        // ---- epilogue: one thread per key --------------------------------------------
+        // ---- epilogue: two threads per key (64 query rows of the tile each) -----------------
         const int quarter = warp & 3;               // TMEM lanes this warp may touch
+        const int hsel = (warp - 2) >> 2;           // which half of the tile's query rows
         const int key_lane = quarter * 32 + lane;
         const int j = kb * kBlk + key_lane;
-        const int et = threadIdx.x - 64;            // 0..127
+        const int et = threadIdx.x - 64;            // 0..255
         const float *lse = a.lse + (size_t)u * a.n;
-        float sum = 0.f;
+        // A failed wait poisons the CTA: later waits return at once and the loop keeps its
+        // shape, so every thread still reaches the final barrier; the status word reports it.
+        auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
+            if (*abort_flag) return false;
+            return mbar_wait(bar, parity, abort_flag);
+        };
         // row constant c_i = lse_i*log2e + (n-1-i)*(-log2 alpha); rows past n give +inf.
         // The value for the NEXT tile is requested one tile ahead so its global-memory latency
-        // never sits between two tiles.
+        // never sits between two tiles.  The lower-half threads publish the 128 constants.
         auto row_const = [&](int i) -> float {
             if (i >= a.n) return INFINITY;
             const int age = a.n - 1 - i;
             return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * a.neg_log2_alpha);
         };
-        float c_next = row_const(kb * kBlk + et);
+        float c_next = hsel == 0 ? row_const(kb * kBlk + et) : 0.f;
+        float sum = 0.f;
         for (int it = 0; it < ntiles; ++it) {
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int i0 = (kb + it) * kBlk;
-            sh->cbuf[it & 1][et] = c_next;
-            mbar_arrive(&sh->c_full[acc]);       // release: the row constants are published
-            if (it + 1 < ntiles) c_next = row_const(i0 + kBlk + et);
-            if (!mbar_wait(&sh->c_full[acc], aph, abort_flag)) break;
-            if (!mbar_wait(&sh->acc_full[acc], aph, abort_flag)) break;
+            if (hsel == 0) sh->cbuf[it & 1][et] = c_next;
+            // every epilogue thread arrives: the constants are published, and nobody is still
+            // reading the buffer that the tile after next will overwrite
+            mbar_arrive(&sh->c_full[acc]);
+            if (hsel == 0 && it + 1 < ntiles) c_next = row_const(i0 + kBlk + et);
+            wait(&sh->c_full[acc], aph);
+            wait(&sh->acc_full[acc], aph);
             tc_fence_after_sync();
-            const float *cb = sh->cbuf[it & 1];
+            const float *cb = sh->cbuf[it & 1] + hsel * 64;
             const bool diag = (it == 0);
-            // the whole 128-row strip of this key comes into registers with one wait, and the
+            // this thread's 64-row strip comes into registers with one wait, and the
             // accumulator buffer goes back to the tensor core before the arithmetic starts
-            uint32_t r[4][32];
-            const uint32_t t_addr = tmem_base + acc * kBlk + ((uint32_t)(quarter * 32) << 16);
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(t_addr + c * 32, r[c]);
+            uint32_t r[2][32];
+            const uint32_t t_addr = tmem_base + acc * kBlk + hsel * 64 + ((uint32_t)(quarter * 32) << 16);
+            tmem_ld32(t_addr, r[0]);
+            tmem_ld32(t_addr + 32, r[1]);
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(&sh->acc_empty[acc]);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 float part = 0.f;
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    float pw = ex2_approx(fmaf(__uint_as_float(r[c][x]), a.sl2, -cb[c * 32 + x]));
-                    if (diag) pw = (i0 + c * 32 + x >= j) ? pw : 0.f;    // causal: rows i >= j
-                    part += pw;
+                for (int x = 0; x < 32; x += 4) {
+                    const float4 c4 = *reinterpret_cast<const float4 *>(cb + c * 32 + x);
+                    const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float pw = ex2_approx(fmaf(__uint_as_float(r[c][x + e]), a.sl2, -cc[e]));
+                        if (diag) pw = (i0 + hsel * 64 + c * 32 + x + e >= j) ? pw : 0.f;   // rows i >= j
+                        part += pw;
+                    }
                 }
                 sum += part;
             }
         }
-        if (j < a.n && !*abort_flag) a.scores[(size_t)u * a.n + j] = sum;
+        if (hsel == 1) sh->part[key_lane] = sum;
+        named_barrier(1, kScoreEpiThreads);
+        if (hsel == 0 && j < a.n && !*abort_flag) a.scores[(size_t)u * a.n + j] = sum + sh->part[key_lane];
     }
 
     tc_fence_before_sync();
