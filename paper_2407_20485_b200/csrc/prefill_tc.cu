@@ -246,27 +246,28 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 // ============================================================================================
 // Attention pass (paper Eq. 3: causal softmax attention):  out_i = sum_j P_ij v_j,  lse_i.
 //
-// One CTA owns 128 query rows (TMEM lanes) and walks the key tiles up to the diagonal.
-//   S = Q K^T          -> TMEM (two buffers, so the next tile's logits are computed while the
-//                         current tile is in the softmax warps)
-//   softmax warps      : one thread per row; running maximum kept lazily (the accumulator is
-//                         rescaled only when the maximum grows by more than 2^8), P rounded to
-//                         the storage type and written back to TENSOR memory, from where the MMA
-//                         reads it as its A operand (shared-memory bandwidth is the scarce
-//                         resource: operands read from it at 128x128x16 per instruction already
-//                         saturate it); the row sum uses the unrounded values
-//   O += P V           -> TMEM; V is consumed as an MN-major operand straight from its TMA tile
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-9
-// softmax + epilogue.  A row is shared by two threads (one per 64-column half): a single
-// warp per scheduler cannot issue the softmax arithmetic fast enough to keep up with the
-// tensor core, two interleaved warps can.  The halves exchange their row maxima through
-// shared memory once per tile and their row sums once at the end.
+// One CTA owns TWO adjacent 128-row query tiles ("streams" A and B) that share every K/V tile.
+// The tensor core alternates between the streams,
+//     S_A(0) S_B(0) | PV_A(0) S_A(1) | PV_B(0) S_B(1) | PV_A(1) S_A(2) | ...
+// so that while one stream's rows are in the softmax warps the other stream's MMAs run.
+//   S = Q K^T        -> TMEM, 128 fp32 columns per stream
+//   softmax warps    : one thread per row.  The running maximum is kept lazily (the accumulator
+//                      is rescaled only when the row maximum grows by more than 2^8).  P, rounded
+//                      to the storage type, is written back into the SAME tensor-memory columns
+//                      the logits came from and is read from there as the A operand of the next
+//                      MMA: shared-memory bandwidth is the scarce resource (two operands read
+//                      from it at 128x128x16 per instruction already saturate it).  The row sum
+//                      uses the unrounded values.
+//   O += P V         -> TMEM, 128 fp32 columns per stream; V is consumed as an MN-major operand
+//                      straight from its TMA tile
+// Tensor memory: S/P_A | O_A | S/P_B | O_B = 512 columns.
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
+// softmax + epilogue of stream A, warps 6-9 of stream B.
 // ============================================================================================
-constexpr int kAttnThreads = 320;            // producer warp, MMA warp, 8 softmax warps
-constexpr int kSoftmaxThreads = 256;
+constexpr int kAttnThreads = 320;
 constexpr int kKStages = 3;                  // K tiles in flight
 constexpr int kVStages = 2;                  // V tiles in flight
-constexpr float kRescaleThreshold = 8.0f;     // log2 units
+constexpr float kRescaleThreshold = 8.0f;    // log2 units
 
 struct AttnArgs {
     void *out;            // [B][H][n][d], strides below
@@ -278,15 +279,13 @@ struct AttnArgs {
 
 struct AttnShared {
     uint64_t q_full, k_full[kKStages], k_empty[kKStages], v_full[kVStages], v_empty[kVStages];
-    uint64_t s_full[2], s_empty[2], p_full, p_empty;
+    uint64_t s_full[2], p_full[2], o_done[2];       // per stream
     uint32_t tmem_base;
     int abort_flag;
-    float xmax[2][2][kBlk];     // [tile parity][column half][row]
-    float lsum[2][kBlk];        // [column half][row]
 };
 
-// Q, K ring, V ring
-constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (1 + kKStages + kVStages) + sizeof(AttnShared);
+// Q_A, Q_B, K ring, V ring
+constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (2 + kKStages + kVStages) + sizeof(AttnShared);
 static_assert(kAttnSmemBytes <= 227 * 1024, "attention pass shared memory");
 
 template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
@@ -302,7 +301,7 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b)
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kAttnThreads)
+__global__ void __launch_bounds__(kAttnThreads, 1)
 attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
 {
@@ -315,8 +314,8 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                 ~uintptr_t(1023));
-    uint8_t *Qs = smem;
-    uint8_t *Ks = smem + kTileBytes;
+    uint8_t *Qs = smem;                                  // two tiles: stream A, stream B
+    uint8_t *Ks = smem + 2 * kTileBytes;
     uint8_t *Vs = Ks + kKStages * kTileBytes;
     AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kVStages * kTileBytes);
 
@@ -326,12 +325,18 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     // split into two bf16 terms (p = hi + lo, |lo| <= 2^-9 |hi|) and both are multiplied
     // with V.  fp16 keeps 11 bits and needs no second term.
     constexpr bool kSplitP = std::is_same<T, __nv_bfloat16>::value;
+
     // CTAs of one unit are adjacent in the grid (longest rows first), so they run together
     // and share the unit's K and V tiles through L2
     const int T_total = (a.n + kBlk - 1) / kBlk;
-    const int u = blockIdx.x / T_total;
-    const int rb = T_total - 1 - blockIdx.x % T_total;
-    const int nt = rb + 1;                              // key tiles 0 .. rb
+    const int npairs = (T_total + 1) / 2;
+    const int u = blockIdx.x / npairs;
+    const int pair = npairs - 1 - blockIdx.x % npairs;
+    const int rbA = 2 * pair, rbB = 2 * pair + 1;
+    const bool hasB = rbB < T_total;
+    const int ntA = rbA + 1;                            // key tiles 0 .. rbA
+    const int ntB = hasB ? rbB + 1 : 0;
+    const int nt = hasB ? ntB : ntA;
     const int b = u / a.H, h = u % a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sh->abort_flag;
@@ -340,9 +345,11 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         mbar_init(&sh->q_full, 1);
         for (int s = 0; s < kKStages; ++s) { mbar_init(&sh->k_full[s], 1); mbar_init(&sh->k_empty[s], 1); }
         for (int s = 0; s < kVStages; ++s) { mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1); }
-        for (int x = 0; x < 2; ++x) { mbar_init(&sh->s_full[x], 1); mbar_init(&sh->s_empty[x], kSoftmaxThreads); }
-        mbar_init(&sh->p_full, kSoftmaxThreads);
-        mbar_init(&sh->p_empty, 1);
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(&sh->s_full[x], 1);
+            mbar_init(&sh->p_full[x], kBlk);
+            mbar_init(&sh->o_done[x], 1);
+        }
         sh->abort_flag = 0;
         fence_mbar_init();
     }
@@ -354,39 +361,45 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sh->tmem_base;
-    // tensor memory columns: S0 | S1 | O | P (high) | P (low)
-    const uint32_t tmem_o = tmem_base + 2 * kBlk;
-    const uint32_t tmem_ph = tmem_base + 3 * kBlk;
-    const uint32_t tmem_pl = tmem_ph + kBlk / 2;
+
+    // A failed wait poisons the CTA: every later wait returns at once, loops keep their shape,
+    // and the status word reports the timeout.
+    auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
+        if (*abort_flag) return false;
+        return mbar_wait(bar, parity, abort_flag);
+    };
 
     if (warp == 0) {
         // ---- TMA producer -------------------------------------------------------------
         if (lane == 0) {
             prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
-            mbar_arrive_expect_tx(&sh->q_full, kTileBytes);
-            tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rb * kBlk, h, b);
-            tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rb * kBlk, h, b);
-            int issued = 0;
+            mbar_arrive_expect_tx(&sh->q_full, hasB ? 2 * kTileBytes : kTileBytes);
+            tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rbA * kBlk, h, b);
+            tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rbA * kBlk, h, b);
+            if (hasB) {
+                tma_load_4d(Qs + kTileBytes, &tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
+                tma_load_4d(Qs + kTileBytes + kHalfBytes, &tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
+            }
+            int k_issued = 0, v_issued = 0;
             for (int t = 0; t < nt; ++t) {
                 const int ks = t % kKStages, vs = t % kVStages;
-                if (!mbar_wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1, abort_flag)) break;
+                if (!wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
                 tma_load_4d(Ks + ks * kTileBytes, &tmap_k, &sh->k_full[ks], 0, t * kBlk, h, b);
                 tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[ks], 64, t * kBlk, h, b);
-                if (!mbar_wait(&sh->v_empty[vs], ((t / kVStages) & 1) ^ 1, abort_flag)) { issued = -(t + 1); break; }
+                k_issued = t + 1;
+                if (!wait(&sh->v_empty[vs], ((t / kVStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->v_full[vs], kTileBytes);
                 tma_load_4d(Vs + vs * kTileBytes, &tmap_v, &sh->v_full[vs], 0, t * kBlk, h, b);
                 tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[vs], 64, t * kBlk, h, b);
-                issued = t + 1;
+                v_issued = t + 1;
             }
             if (*abort_flag) {
                 // bounded chance for copies in flight to land before the CTA exits
                 int dummy = 0;
-                const int kdone = issued < 0 ? -issued : issued;
-                const int vdone = issued < 0 ? -issued - 1 : issued;
-                for (int t = max(0, kdone - kKStages); t < kdone; ++t)
+                for (int t = max(0, k_issued - kKStages); t < k_issued; ++t)
                     mbar_wait(&sh->k_full[t % kKStages], (t / kKStages) & 1, &dummy);
-                for (int t = max(0, vdone - kVStages); t < vdone; ++t)
+                for (int t = max(0, v_issued - kVStages); t < v_issued; ++t)
                     mbar_wait(&sh->v_full[t % kVStages], (t / kVStages) & 1, &dummy);
                 mbar_wait(&sh->q_full, 0, &dummy);
             }
@@ -397,179 +410,186 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
             const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
             const uint32_t q_addr = smem_u32(Qs);
-            auto issue_s = [&](int t) -> bool {
-                const int s = t % kKStages;
-                const int sb = t & 1;
-                if (!mbar_wait(&sh->k_full[s], (t / kKStages) & 1, abort_flag)) return false;
-                if (!mbar_wait(&sh->s_empty[sb], ((t >> 1) & 1) ^ 1, abort_flag)) return false;
-                tc_fence_after_sync();
-                issue_qk_mma(tmem_base + sb * kBlk, q_addr, smem_u32(Ks + s * kTileBytes), idesc_qk);
-                umma_commit(&sh->k_empty[s]);
-                umma_commit(&sh->s_full[sb]);
-                return true;
+            // S_X(t) = Q_X K_t^T into stream X's logits columns
+            auto issue_s = [&](int X, int t) {
+                issue_qk_mma(tmem_base + X * 2 * kBlk, q_addr + X * kTileBytes,
+                             smem_u32(Ks + (t % kKStages) * kTileBytes), idesc_qk);
+                umma_commit(&sh->s_full[X]);
             };
-            bool ok = mbar_wait(&sh->q_full, 0, abort_flag);
-            ok = ok && issue_s(0);
-            for (int t = 0; ok && t < nt; ++t) {
-                if (t + 1 < nt && !issue_s(t + 1)) break;
-                const int s = t % kVStages;
-                if (!mbar_wait(&sh->p_full, t & 1, abort_flag)) break;
-                if (!mbar_wait(&sh->v_full[s], (t / kVStages) & 1, abort_flag)) break;
-                tc_fence_after_sync();
-                const uint32_t v_addr = smem_u32(Vs + s * kTileBytes);
+            // O_X += P_X(t) V_t with P read from stream X's logits columns
+            auto issue_pv = [&](int X, int t) {
+                const uint32_t v_addr = smem_u32(Vs + (t % kVStages) * kTileBytes);
+                const uint32_t sp = tmem_base + X * 2 * kBlk, o = sp + kBlk;
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k) {
-                    // A = P from tensor memory: 16 keys = 8 columns; B = V: 16 keys = two 8-row
-                    // groups of 1024 bytes, the two 64-wide d halves 16 KB apart
+                    // 16 keys: 8 columns of packed P; V: two 8-row groups of 1024 bytes, the two
+                    // 64-wide d halves 16 KB apart
                     const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                    umma_ts(tmem_o, tmem_ph + k * 8, bdesc, idesc_pv, (t > 0) || (k > 0));
+                    umma_ts(o, sp + k * 8, bdesc, idesc_pv, (t > 0) || (k > 0));
                 }
                 if (kSplitP) {
 #pragma unroll
                     for (int k = 0; k < kBlk / 16; ++k) {
                         const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                        umma_ts(tmem_o, tmem_pl + k * 8, bdesc, idesc_pv, 1);
+                        umma_ts(o, sp + kBlk / 2 + k * 8, bdesc, idesc_pv, 1);
                     }
                 }
-                umma_commit(&sh->v_empty[s]);
-                umma_commit(&sh->p_empty);
+                umma_commit(&sh->o_done[X]);
+            };
+            wait(&sh->q_full, 0);
+            wait(&sh->k_full[0], 0);
+            tc_fence_after_sync();
+            issue_s(0, 0);
+            if (hasB) issue_s(1, 0);
+            umma_commit(&sh->k_empty[0]);
+            for (int t = 0; t < nt; ++t) {
+                const bool nextA = t + 1 < ntA, nextB = t + 1 < ntB;
+                wait(&sh->v_full[t % kVStages], (t / kVStages) & 1);
+                if (nextA || nextB) wait(&sh->k_full[(t + 1) % kKStages], ((t + 1) / kKStages) & 1);
+                if (t < ntA) {
+                    wait(&sh->p_full[0], t & 1);
+                    tc_fence_after_sync();
+                    issue_pv(0, t);
+                    if (nextA) issue_s(0, t + 1);
+                }
+                if (t < ntB) {
+                    wait(&sh->p_full[1], t & 1);
+                    tc_fence_after_sync();
+                    issue_pv(1, t);
+                    if (nextB) issue_s(1, t + 1);
+                }
+                umma_commit(&sh->v_empty[t % kVStages]);
+                if (nextA || nextB) umma_commit(&sh->k_empty[(t + 1) % kKStages]);
             }
         }
     } else {
-        // ---- softmax + epilogue: two threads per query row (64 columns each) ---------------
+        // ---- softmax + epilogue: one thread per query row of its stream --------------------
+        const int X = (warp - 2) >> 2;                     // stream
+        const int ntX = X == 0 ? ntA : ntB;
         const int quarter = warp & 3;                      // TMEM lanes this warp may touch
-        const int hsel = (warp - 2) >> 2;                  // column half
         const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
-        const int i = rb * kBlk + r;
+        const int i = (X == 0 ? rbA : rbB) * kBlk + r;
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-        const int col0 = hsel * 64;
-        // A failed wait poisons the CTA: later waits return at once, the loop keeps its shape
-        // (so every thread still meets the named barrier) and the status word reports it.
-        auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
-            if (*abort_flag) return false;
-            return mbar_wait(bar, parity, abort_flag);
-        };
+        const uint32_t sp = tmem_base + X * 2 * kBlk + lane_off;   // logits, then P hi | P lo
+        const uint32_t to = sp + kBlk;                             // output accumulator
         float m_used = 0.f, l = 0.f;
-        for (int t = 0; t < nt; ++t) {
-            const int sb = t & 1;
-            wait(&sh->s_full[sb], (t >> 1) & 1);
+        for (int t = 0; t < ntX; ++t) {
+            wait(&sh->s_full[X], t & 1);
             tc_fence_after_sync();
-            const uint32_t s_addr = tmem_base + sb * kBlk + lane_off + col0;
-            const bool diag = (t == nt - 1);
-            // this thread's half of the logits row comes into registers with one wait
-            uint32_t v[2][32];
-            tmem_ld32(s_addr, v[0]);
-            tmem_ld32(s_addr + 32, v[1]);
-            tmem_wait_ld();
-            tc_fence_before_sync();
-            mbar_arrive(&sh->s_empty[sb]);
-            // exponent arguments relative to the current reference maximum (log2 domain)
-            float xmax = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 2; ++c)
+            const bool diag = (t == ntX - 1);
+            // pass 1: row maximum of the raw logits
+            float smax = -INFINITY;
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(sp + c * 32, v);
+                tmem_wait_ld();
 #pragma unroll
                 for (int x = 0; x < 32; ++x) {
-                    float e = fmaf(__uint_as_float(v[c][x]), a.sl2, -m_used);
-                    if (diag && col0 + c * 32 + x > r) e = -INFINITY;     // causal mask
-                    xmax = fmaxf(xmax, e);
-                    v[c][x] = __float_as_uint(e);
+                    float sv = __uint_as_float(v[x]);
+                    if (diag && c * 32 + x > r) sv = -INFINITY;           // causal mask
+                    smax = fmaxf(smax, sv);
                 }
-            sh->xmax[t & 1][hsel][r] = xmax;
-            named_barrier(1, kSoftmaxThreads);
-            xmax = fmaxf(xmax, sh->xmax[t & 1][hsel ^ 1][r]);
-            // Lazy maximum: the reference moves only on the first tile or when the row maximum
-            // exceeds it by more than 2^8; otherwise probabilities up to 256 are simply kept.
-            float factor = 1.f;
+            }
+            // Lazy maximum (log2 domain): the reference moves only on the first tile or when
+            // the row maximum exceeds it by more than 2^8; otherwise probabilities up to 256
+            // are simply kept.
+            const float xmax = fmaf(smax, a.sl2, -m_used);
             const bool grow = (t == 0) || (xmax > kRescaleThreshold);
+            float factor = 1.f;
             if (grow) {
                 m_used += xmax;
                 factor = t == 0 ? 0.f : ex2_approx(-xmax);
             }
-            float rowsum = 0.f;
-            if (__any_sync(0xffffffffu, grow)) {
-                const float shift = grow ? xmax : 0.f;
-#pragma unroll
-                for (int c = 0; c < 2; ++c)
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const float pv = ex2_approx(__uint_as_float(v[c][x]) - shift);   // masked -> 0
-                        rowsum += pv;
-                        v[c][x] = __float_as_uint(pv);
-                    }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 2; ++c)
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        const float pv = ex2_approx(__uint_as_float(v[c][x]));
-                        rowsum += pv;
-                        v[c][x] = __float_as_uint(pv);
-                    }
-            }
-            l = fmaf(l, factor, rowsum);
-            // P(t-1) has been consumed and O holds tiles 0..t-1 once p_empty completes
-            if (t > 0) wait(&sh->p_empty, (t - 1) & 1);
-            tc_fence_after_sync();
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
+                // O_X holds tiles 0..t-1 once the previous P V product has retired
+                wait(&sh->o_done[X], (t - 1) & 1);
+                tc_fence_after_sync();
 #pragma unroll 1
-                for (int c = 0; c < 2; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
-                    tmem_ld32(tmem_o + lane_off + col0 + c * 32, o);
+                    tmem_ld32(to + c * 32, o);
                     tmem_wait_ld();
 #pragma unroll
                     for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * factor);
-                    tmem_st32(tmem_o + lane_off + col0 + c * 32, o);
+                    tmem_st32(to + c * 32, o);
                 }
                 tmem_wait_st();
             }
-            // P (rounded to the storage type; for bf16 also the rounding remainder) to tensor
-            // memory: two 16-bit values per 32-bit column, 32 keys = 16 columns
+            // pass 2: probabilities; P overwrites the logits columns.  32 logits columns become
+            // 16 columns of P (high part at [16c, 16c+16), low part at [64+16c, 80+16c)).  The
+            // high part only lands on columns already read; the low parts of the first three
+            // chunks are held back until their destination columns have been read.
+            const float neg_m = -m_used;
+            float rowsum = 0.f;
+            uint32_t lo_hold[3][16];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < 4; ++c) {
+                uint32_t v[32];
+                tmem_ld32(sp + c * 32, v);
+                tmem_wait_ld();
                 uint32_t hi[16], lo[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float p0 = __uint_as_float(v[c][2 * e]);
-                    const float p1 = __uint_as_float(v[c][2 * e + 1]);
+                    float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * e]), a.sl2, neg_m));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * e + 1]), a.sl2, neg_m));
+                    if (diag) {
+                        if (c * 32 + 2 * e > r) p0 = 0.f;
+                        if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
+                    }
+                    rowsum += p0 + p1;
                     hi[e] = pack2<T>(p0, p1);
                     if (kSplitP)      // a bf16 is the upper half of an fp32
                         lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
                                          p1 - __uint_as_float(hi[e] & 0xffff0000u));
                 }
-                tmem_st16(tmem_ph + lane_off + (hsel * 2 + c) * 16, hi);
-                if (kSplitP) tmem_st16(tmem_pl + lane_off + (hsel * 2 + c) * 16, lo);
-            }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            mbar_arrive(&sh->p_full);
-        }
-        // ---- epilogue ---------------------------------------------------------------------
-        sh->lsum[hsel][r] = l;
-        named_barrier(1, kSoftmaxThreads);
-        l += sh->lsum[hsel ^ 1][r];
-        const bool done = wait(&sh->p_empty, (nt - 1) & 1);
-        tc_fence_after_sync();
-        if (done) {
-            const float inv = 1.f / l;
-            T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t + col0;
-#pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tmem_o + lane_off + col0 + c * 32, o);
-                tmem_wait_ld();
-                if (i < a.n) {
+                tmem_st16(sp + c * 16, hi);
+                if (kSplitP) {
+                    if (c < 3) {
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            w[e] = pack2<T>(__uint_as_float(o[q4 * 8 + 2 * e]) * inv,
-                                            __uint_as_float(o[q4 * 8 + 2 * e + 1]) * inv);
-                        *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        for (int e = 0; e < 16; ++e) lo_hold[c][e] = lo[e];
+                    }
+                    if (c == 2) {            // columns 64..95 have been read
+                        tmem_st16(sp + 64, lo_hold[0]);
+                        tmem_st16(sp + 80, lo_hold[1]);
+                    }
+                    if (c == 3) {            // columns 96..127 have been read
+                        tmem_st16(sp + 96, lo_hold[2]);
+                        tmem_st16(sp + 112, lo);
                     }
                 }
             }
-            if (i < a.n && hsel == 0) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
+            tmem_wait_st();
+            l = fmaf(l, factor, rowsum);
+            tc_fence_before_sync();
+            mbar_arrive(&sh->p_full[X]);
+        }
+        // ---- epilogue ---------------------------------------------------------------------
+        if (ntX > 0) {
+            const bool done = wait(&sh->o_done[X], (ntX - 1) & 1);
+            tc_fence_after_sync();
+            if (done) {
+                const float inv = 1.f / l;
+                T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t;
+#pragma unroll 1
+                for (int c = 0; c < kD / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(to + c * 32, o);
+                    tmem_wait_ld();
+                    if (i < a.n) {
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                w[e] = pack2<T>(__uint_as_float(o[q4 * 8 + 2 * e]) * inv,
+                                                __uint_as_float(o[q4 * 8 + 2 * e + 1]) * inv);
+                            *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    }
+                }
+                if (i < a.n) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
+            }
         }
     }
 
@@ -648,7 +668,8 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
     aa.n = a.n; aa.H = a.H;
     aa.sl2 = a.scale * kLog2e;
-    const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
+    const int npairs = ((a.n + kBlk - 1) / kBlk + 1) / 2;
+    const dim3 grid((unsigned)((size_t)a.B * a.H * npairs));
     if (dtype == A2SF_BF16)
         attn_pass_tc<__nv_bfloat16><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
     else
