@@ -59,16 +59,22 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
-// 8 K-steps of 16 elements over a [128 x 128] K-major operand pair stored as two
-// 64-column swizzled halves.
-__device__ __forceinline__ void issue_qk_mma(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr,
+// The issuing thread is the bottleneck of small-tile UMMA pipelines, so descriptors are built
+// once per operand buffer and only advanced by a constant per K-step.
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t smem_addr)
+{
+    return make_sdesc_sw128(smem_addr, 16, 1024);
+}
+
+// 8 K-steps of 16 elements over a [128 x 128] K-major operand pair stored as two 64-column
+// swizzled halves: step k starts (k/4) halves + (k%4)*32 bytes into the tile (16-byte units).
+__device__ __forceinline__ void issue_qk_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                              uint32_t idesc)
 {
 #pragma unroll
     for (int k = 0; k < kD / 16; ++k) {
-        const uint32_t off = (k >> 2) * kHalfBytes + (k & 3) * 32;
-        umma_ss(d_tmem, make_sdesc_sw128(a_addr + off, 16, 1024),
-                make_sdesc_sw128(b_addr + off, 16, 1024), idesc, k > 0);
+        const uint64_t off = (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
+        umma_ss(d_tmem, a_desc + off, b_desc + off, idesc, k > 0);
     }
 }
 
@@ -149,7 +155,9 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         // ---- MMA issuer -------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
-            const uint32_t k_addr = smem_u32(Ks);
+            const uint64_t k_desc = kmajor_desc(smem_u32(Ks));
+            uint64_t q_desc[kScoreStages];
+            for (int s = 0; s < kScoreStages; ++s) q_desc[s] = kmajor_desc(smem_u32(Qs + s * kTileBytes));
             bool ok = mbar_wait(&sh->k_full, 0, abort_flag);
             for (int it = 0; ok && it < ntiles; ++it) {
                 const int s = it % kScoreStages;
@@ -159,7 +167,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
                 if (!mbar_wait(&sh->q_full[s], ph, abort_flag)) break;
                 if (!mbar_wait(&sh->acc_empty[acc], aph ^ 1, abort_flag)) break;
                 tc_fence_after_sync();
-                issue_qk_mma(tmem_base + acc * kBlk, k_addr, smem_u32(Qs + s * kTileBytes), idesc);
+                issue_qk_mma(tmem_base + acc * kBlk, k_desc, q_desc[s], idesc);
                 umma_commit(&sh->q_empty[s]);       // the stage is free once these MMAs retire
                 umma_commit(&sh->acc_full[acc]);
             }
@@ -409,30 +417,29 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
             const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
-            const uint32_t q_addr = smem_u32(Qs);
+            uint64_t q_desc[2], k_desc[kKStages], v_desc[kVStages];
+            for (int x = 0; x < 2; ++x) q_desc[x] = kmajor_desc(smem_u32(Qs + x * kTileBytes));
+            for (int x = 0; x < kKStages; ++x) k_desc[x] = kmajor_desc(smem_u32(Ks + x * kTileBytes));
+            // V as an MN-major operand: 64-wide d halves 16 KB apart, 8-key groups 1024 bytes apart
+            for (int x = 0; x < kVStages; ++x)
+                v_desc[x] = make_sdesc_sw128(smem_u32(Vs + x * kTileBytes), kHalfBytes, 1024);
             // S_X(t) = Q_X K_t^T into stream X's logits columns
             auto issue_s = [&](int X, int t) {
-                issue_qk_mma(tmem_base + X * 2 * kBlk, q_addr + X * kTileBytes,
-                             smem_u32(Ks + (t % kKStages) * kTileBytes), idesc_qk);
+                issue_qk_mma(tmem_base + X * 2 * kBlk, q_desc[X], k_desc[t % kKStages], idesc_qk);
                 umma_commit(&sh->s_full[X]);
             };
             // O_X += P_X(t) V_t with P read from stream X's logits columns
             auto issue_pv = [&](int X, int t) {
-                const uint32_t v_addr = smem_u32(Vs + (t % kVStages) * kTileBytes);
+                const uint64_t vd = v_desc[t % kVStages];
                 const uint32_t sp = tmem_base + X * 2 * kBlk, o = sp + kBlk;
+                // 16 keys per step: 8 columns of packed P; two 8-key groups of V = 2048 bytes
 #pragma unroll
-                for (int k = 0; k < kBlk / 16; ++k) {
-                    // 16 keys: 8 columns of packed P; V: two 8-row groups of 1024 bytes, the two
-                    // 64-wide d halves 16 KB apart
-                    const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                    umma_ts(o, sp + k * 8, bdesc, idesc_pv, (t > 0) || (k > 0));
-                }
+                for (int k = 0; k < kBlk / 16; ++k)
+                    umma_ts(o, sp + k * 8, vd + (uint64_t)(k * 2048 >> 4), idesc_pv, (t > 0) || (k > 0));
                 if (kSplitP) {
 #pragma unroll
-                    for (int k = 0; k < kBlk / 16; ++k) {
-                        const uint64_t bdesc = make_sdesc_sw128(v_addr + k * 2048, kHalfBytes, 1024);
-                        umma_ts(o, sp + kBlk / 2 + k * 8, bdesc, idesc_pv, 1);
-                    }
+                    for (int k = 0; k < kBlk / 16; ++k)
+                        umma_ts(o, sp + kBlk / 2 + k * 8, vd + (uint64_t)(k * 2048 >> 4), idesc_pv, 1);
                 }
                 umma_commit(&sh->o_done[X]);
             };
