@@ -484,20 +484,23 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             wait(&sh->s_full[X], t & 1);
             tc_fence_after_sync();
             const bool diag = (t == ntX - 1);
-            // pass 1: row maximum of the raw logits
+            // pass 1: row maximum of the raw logits.  Only the diagonal tile pays for the mask.
             float smax = -INFINITY;
+            auto row_max = [&](auto masked) {
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(sp + c * 32, v);
-                tmem_wait_ld();
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(sp + c * 32, v);
+                    tmem_wait_ld();
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    float sv = __uint_as_float(v[x]);
-                    if (diag && c * 32 + x > r) sv = -INFINITY;           // causal mask
-                    smax = fmaxf(smax, sv);
+                    for (int x = 0; x < 32; ++x) {
+                        float sv = __uint_as_float(v[x]);
+                        if (decltype(masked)::value && c * 32 + x > r) sv = -INFINITY;   // causal mask
+                        smax = fmaxf(smax, sv);
+                    }
                 }
-            }
+            };
+            if (diag) row_max(std::true_type{}); else row_max(std::false_type{});
             // Lazy maximum (log2 domain): the reference moves only on the first tile or when
             // the row maximum exceeds it by more than 2^8; otherwise probabilities up to 256
             // are simply kept.
@@ -529,43 +532,46 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             // chunks are held back until their destination columns have been read.
             const float neg_m = -m_used;
             float rowsum = 0.f;
-            uint32_t lo_hold[3][16];
+            auto write_p = [&](auto masked) {
+                uint32_t lo_hold[3][16];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t v[32];
-                tmem_ld32(sp + c * 32, v);
-                tmem_wait_ld();
-                uint32_t hi[16], lo[16];
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(sp + c * 32, v);
+                    tmem_wait_ld();
+                    uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * e]), a.sl2, neg_m));
-                    float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * e + 1]), a.sl2, neg_m));
-                    if (diag) {
-                        if (c * 32 + 2 * e > r) p0 = 0.f;
-                        if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
+                    for (int e = 0; e < 16; ++e) {
+                        float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * e]), a.sl2, neg_m));
+                        float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * e + 1]), a.sl2, neg_m));
+                        if (decltype(masked)::value) {
+                            if (c * 32 + 2 * e > r) p0 = 0.f;
+                            if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
+                        }
+                        rowsum += p0 + p1;
+                        hi[e] = pack2<T>(p0, p1);
+                        if (kSplitP)      // a bf16 is the upper half of an fp32
+                            lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
+                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
                     }
-                    rowsum += p0 + p1;
-                    hi[e] = pack2<T>(p0, p1);
-                    if (kSplitP)      // a bf16 is the upper half of an fp32
-                        lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
-                                         p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    tmem_st16(sp + c * 16, hi);
+                    if (kSplitP) {
+                        if (c < 3) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) lo_hold[c][e] = lo[e];
+                        }
+                        if (c == 2) {            // columns 64..95 have been read
+                            tmem_st16(sp + 64, lo_hold[0]);
+                            tmem_st16(sp + 80, lo_hold[1]);
+                        }
+                        if (c == 3) {            // columns 96..127 have been read
+                            tmem_st16(sp + 96, lo_hold[2]);
+                            tmem_st16(sp + 112, lo);
+                        }
+                    }
                 }
-                tmem_st16(sp + c * 16, hi);
-                if (kSplitP) {
-                    if (c < 3) {
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) lo_hold[c][e] = lo[e];
-                    }
-                    if (c == 2) {            // columns 64..95 have been read
-                        tmem_st16(sp + 64, lo_hold[0]);
-                        tmem_st16(sp + 80, lo_hold[1]);
-                    }
-                    if (c == 3) {            // columns 96..127 have been read
-                        tmem_st16(sp + 96, lo_hold[2]);
-                        tmem_st16(sp + 112, lo);
-                    }
-                }
-            }
+            };
+            if (diag) write_p(std::true_type{}); else write_p(std::false_type{});
             tmem_wait_st();
             l = fmaf(l, factor, rowsum);
             tc_fence_before_sync();
