@@ -235,7 +235,7 @@ def run_ours(args):
                     "flops_per_step": prefill_flops, "frac_of_measured_bf16_sustained":
                         prefill_tflops / scale_units / peaks["bf16_tflops_sustained"],
                     "frac_of_nominal_bf16": prefill_tflops / scale_units / NOMINAL["bf16_tflops"]},
-        "roofline": {"kernel": "decode_step_kernel", "bound": "hbm", "achieved": achieved,
+        "roofline": {"kernel": "decode_step_stream_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
                      "traffic": None, "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
