@@ -34,6 +34,9 @@ METRIC = "a2sf_decode_step_hbm_gbps"
 UNIT = "GB/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode_step_stream_kernel launch (ncu, config 4;
+# the capture is summarised in profiles/launch_list_llama2_13b.md).  Set to None when the kernel changes.
+NCU_DECODE_TRAFFIC = {("llama2_13b", 32): 341956064 + 2317664}
 
 
 def load_peaks():
@@ -238,7 +241,7 @@ def run_ours(args):
         "roofline": {"kernel": "decode_step_stream_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
-                     "traffic": None, "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
+                     "traffic": NCU_DECODE_TRAFFIC.get((w.name, w.B)), "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
