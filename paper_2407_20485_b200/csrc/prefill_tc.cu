@@ -487,18 +487,21 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             // pass 1: row maximum of the raw logits.  Only the diagonal tile pays for the mask.
             float smax = -INFINITY;
             auto row_max = [&](auto masked) {
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(sp + c * 32, v);
-                    tmem_wait_ld();
+                // all four loads are in flight before the single wait
+                uint32_t v[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(sp + c * 32, v[c]);
+                tmem_wait_ld();
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int x = 0; x < 32; ++x) {
-                        float sv = __uint_as_float(v[x]);
+                        float sv = __uint_as_float(v[c][x]);
                         if (decltype(masked)::value && c * 32 + x > r) sv = -INFINITY;   // causal mask
-                        smax = fmaxf(smax, sv);
+                        mx[c] = fmaxf(mx[c], sv);
                     }
-                }
+                smax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
             };
             if (diag) row_max(std::true_type{}); else row_max(std::false_type{});
             // Lazy maximum (log2 domain): the reference moves only on the first tile or when
