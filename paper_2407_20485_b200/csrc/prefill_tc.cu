@@ -259,10 +259,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //     S_A(0) S_B(0) | PV_A(0) S_A(1) | PV_B(0) S_B(1) | PV_A(1) S_A(2) | ...
 // so that while one stream's rows are in the softmax warps the other stream's MMAs run.
 //   S = Q K^T        -> TMEM, 128 fp32 columns per stream
-//   softmax warps    : two threads per row, one per 64-column half (a single warp per scheduler
-//                      cannot issue the softmax arithmetic fast enough; the halves exchange their
-//                      row maxima through shared memory once per tile and their row sums at the
-//                      end).  The running maximum is kept lazily (the accumulator
+//   softmax warps    : one thread per row.  The running maximum is kept lazily (the accumulator
 //                      is rescaled only when the row maximum grows by more than 2^8).  P, rounded
 //                      to the storage type, is written back into the SAME tensor-memory columns
 //                      the logits came from and is read from there as the A operand of the next
@@ -272,11 +269,11 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //   O += P V         -> TMEM, 128 fp32 columns per stream; V is consumed as an MN-major operand
 //                      straight from its TMA tile
 // Tensor memory: S/P_A | O_A | S/P_B | O_B = 512 columns.
-// Warp roles (576 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-9
-// softmax + epilogue of stream A, warps 10-17 of stream B.
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
+// softmax + epilogue of stream A, warps 6-9 of stream B.
 // ============================================================================================
-constexpr int kAttnThreads = 576;            // producer, MMA issuer, 2 streams x 8 softmax warps
-constexpr int kKStages = 2;                  // K tiles in flight
+constexpr int kAttnThreads = 320;
+constexpr int kKStages = 3;                  // K tiles in flight
 constexpr int kVStages = 2;                  // V tiles in flight
 constexpr float kRescaleThreshold = 8.0f;    // log2 units
 
@@ -293,8 +290,6 @@ struct AttnShared {
     uint64_t s_full[2], p_full[2], o_done[2];       // per stream
     uint32_t tmem_base;
     int abort_flag;
-    float xmax[2][2][2][kBlk];  // [stream][tile parity][column half][row]
-    float lsum[2][2][kBlk];     // [stream][column half][row]
 };
 
 // Q_A, Q_B, K ring, V ring
@@ -360,7 +355,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         for (int s = 0; s < kVStages; ++s) { mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1); }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sh->s_full[x], 1);
-            mbar_init(&sh->p_full[x], 2 * kBlk);
+            mbar_init(&sh->p_full[x], kBlk);
             mbar_init(&sh->o_done[x], 1);
         }
         sh->abort_flag = 0;
@@ -475,45 +470,40 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             }
         }
     } else {
-        // ---- softmax + epilogue: two threads per query row of a stream (64 columns each) ----
-        const int X = (warp - 2) >> 3;                     // stream: warps 2-9 = A, 10-17 = B
-        const int hsel = ((warp - 2) >> 2) & 1;            // column half
+        // ---- softmax + epilogue: one thread per query row of its stream --------------------
+        const int X = (warp - 2) >> 2;                     // stream
         const int ntX = X == 0 ? ntA : ntB;
         const int quarter = warp & 3;                      // TMEM lanes this warp may touch
         const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
         const int i = (X == 0 ? rbA : rbB) * kBlk + r;
-        const int col0 = hsel * 64;
         const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
         const uint32_t sp = tmem_base + X * 2 * kBlk + lane_off;   // logits, then P hi | P lo
-        const uint32_t to = sp + kBlk + col0;                      // this thread's half of O
+        const uint32_t to = sp + kBlk;                             // output accumulator
         float m_used = 0.f, l = 0.f;
         for (int t = 0; t < ntX; ++t) {
             wait(&sh->s_full[X], t & 1);
             tc_fence_after_sync();
             const bool diag = (t == ntX - 1);
-            // this thread's 64 logits come into registers once and stay there
-            uint32_t v[2][32];
-            tmem_ld32(sp + col0, v[0]);
-            tmem_ld32(sp + col0 + 32, v[1]);
-            tmem_wait_ld();
-            float mx0 = -INFINITY, mx1 = -INFINITY;
-            if (diag) {
+            // pass 1: row maximum of the raw logits.  Only the diagonal tile pays for the mask.
+            float smax = -INFINITY;
+            auto row_max = [&](auto masked) {
+                // all four loads are in flight before the single wait
+                uint32_t v[4][32];
 #pragma unroll
-                for (int x = 0; x < 32; ++x) {
-                    if (col0 + x > r) v[0][x] = 0xff800000u;             // causal mask: -inf
-                    if (col0 + 32 + x > r) v[1][x] = 0xff800000u;
-                }
-            }
+                for (int c = 0; c < 4; ++c) tmem_ld32(sp + c * 32, v[c]);
+                tmem_wait_ld();
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int x = 0; x < 32; ++x) {
-                mx0 = fmaxf(mx0, __uint_as_float(v[0][x]));
-                mx1 = fmaxf(mx1, __uint_as_float(v[1][x]));
-            }
-            // The halves exchange their maxima.  Passing this barrier also means both halves
-            // hold their logits in registers, so P may now overwrite the logits columns.
-            sh->xmax[X][t & 1][hsel][r] = fmaxf(mx0, mx1);
-            named_barrier(1 + X, 2 * kBlk);
-            const float smax = fmaxf(fmaxf(mx0, mx1), sh->xmax[X][t & 1][hsel ^ 1][r]);
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) {
+                        float sv = __uint_as_float(v[c][x]);
+                        if (decltype(masked)::value && c * 32 + x > r) sv = -INFINITY;   // causal mask
+                        mx[c] = fmaxf(mx[c], sv);
+                    }
+                smax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            };
+            if (diag) row_max(std::true_type{}); else row_max(std::false_type{});
             // Lazy maximum (log2 domain): the reference moves only on the first tile or when
             // the row maximum exceeds it by more than 2^8; otherwise probabilities up to 256
             // are simply kept.
@@ -529,7 +519,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 wait(&sh->o_done[X], (t - 1) & 1);
                 tc_fence_after_sync();
 #pragma unroll 1
-                for (int c = 0; c < 2; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(to + c * 32, o);
                     tmem_wait_ld();
@@ -539,28 +529,52 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 }
                 tmem_wait_st();
             }
-            // probabilities; P (rounded to the storage type, for bf16 also the rounding
-            // remainder) overwrites the logits columns: 32 logits columns become 16 columns of
-            // the high part at [16g, 16g+16) and 16 of the low part at [64+16g, 80+16g)
+            // pass 2: probabilities; P overwrites the logits columns.  32 logits columns become
+            // 16 columns of P (high part at [16c, 16c+16), low part at [64+16c, 80+16c)).  The
+            // high part only lands on columns already read; the low parts of the first three
+            // chunks are held back until their destination columns have been read.
             const float neg_m = -m_used;
             float rowsum = 0.f;
+            auto write_p = [&](auto masked) {
+                uint32_t lo_hold[3][16];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t hi[16], lo[16];
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(sp + c * 32, v);
+                    tmem_wait_ld();
+                    uint32_t hi[16], lo[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e]), a.sl2, neg_m));      // masked -> 0
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e + 1]), a.sl2, neg_m));
-                    rowsum += p0 + p1;
-                    hi[e] = pack2<T>(p0, p1);
-                    if (kSplitP)      // a bf16 is the upper half of an fp32
-                        lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
-                                         p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    for (int e = 0; e < 16; ++e) {
+                        float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * e]), a.sl2, neg_m));
+                        float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * e + 1]), a.sl2, neg_m));
+                        if (decltype(masked)::value) {
+                            if (c * 32 + 2 * e > r) p0 = 0.f;
+                            if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
+                        }
+                        rowsum += p0 + p1;
+                        hi[e] = pack2<T>(p0, p1);
+                        if (kSplitP)      // a bf16 is the upper half of an fp32
+                            lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
+                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    }
+                    tmem_st16(sp + c * 16, hi);
+                    if (kSplitP) {
+                        if (c < 3) {
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) lo_hold[c][e] = lo[e];
+                        }
+                        if (c == 2) {            // columns 64..95 have been read
+                            tmem_st16(sp + 64, lo_hold[0]);
+                            tmem_st16(sp + 80, lo_hold[1]);
+                        }
+                        if (c == 3) {            // columns 96..127 have been read
+                            tmem_st16(sp + 96, lo_hold[2]);
+                            tmem_st16(sp + 112, lo);
+                        }
+                    }
                 }
-                const int g = hsel * 2 + c;
-                tmem_st16(sp + g * 16, hi);
-                if (kSplitP) tmem_st16(sp + 64 + g * 16, lo);
-            }
+            };
+            if (diag) write_p(std::true_type{}); else write_p(std::false_type{});
             tmem_wait_st();
             l = fmaf(l, factor, rowsum);
             tc_fence_before_sync();
@@ -568,17 +582,13 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         }
         // ---- epilogue ---------------------------------------------------------------------
         if (ntX > 0) {
-            sh->lsum[X][hsel][r] = l;
-            named_barrier(1 + X, 2 * kBlk);
-            l += sh->lsum[X][hsel ^ 1][r];
             const bool done = wait(&sh->o_done[X], (ntX - 1) & 1);
             tc_fence_after_sync();
             if (done) {
                 const float inv = 1.f / l;
-                T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h +
-                          (int64_t)i * a.st_t + col0;
+                T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t;
 #pragma unroll 1
-                for (int c = 0; c < 2; ++c) {
+                for (int c = 0; c < kD / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(to + c * 32, o);
                     tmem_wait_ld();
@@ -594,7 +604,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                         }
                     }
                 }
-                if (i < a.n && hsel == 0) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
+                if (i < a.n) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
         }
     }
