@@ -5,10 +5,14 @@
 //
 // Memory-bound: every K and V row of the head is read exactly once with 16-byte
 // loads, lanes laid across the row so a warp reads whole 512-byte spans.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "tc_sm100.cuh"
 
 namespace a2sf {
+
+namespace cg = cooperative_groups;
 
 // sticky device-side status of the decode kernels (a bounded wait that ran out)
 static __device__ int g_decode_status = 0;
@@ -26,6 +30,7 @@ int *decode_status_word()
 }
 
 constexpr int kDecodeThreads = 256;
+constexpr int kSplitMinBudget = 512;         // split-K only pays for long caches
 constexpr int kUnroll = 4;
 
 template <int NT>
@@ -54,30 +59,59 @@ __device__ __forceinline__ float block_sum(float v, float *red)
     return r;
 }
 
+// ============================================================================================
+// Split-K variant for few units with large budgets (flash-decoding): a thread-block cluster of
+// C CTAs shares one unit, each CTA owning a contiguous slice of its slots.  Every CTA computes
+// the logits, the local maximum, the local exponential sum and the unnormalised partial output
+// of its slice; the partials meet in distributed shared memory: all CTAs read every (max, sum)
+// pair to form the global softmax constants, rank 0 combines the partial outputs, every CTA
+// then updates the scores of its own slots and publishes its local eviction candidate, and
+// rank 0 picks the global (score, position) minimum and writes the new token in place.
+// With C = 1 this is the plain one-CTA-per-unit kernel.
+// ============================================================================================
+struct SplitExchange {
+    float m, l;                    // local maximum and sum of exp(logit - m)
+    unsigned long long best;       // local (bits(S) << 32 | position) minimum over evictable slots
+    int best_slot;
+    float out[128];                // unnormalised partial output (relative to m)
+};
+
 template <typename T, int D, int NT>
 __global__ void __launch_bounds__(NT)
-decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *__restrict__ k_new,
-                   const T *__restrict__ v_new, T *__restrict__ out, int32_t *__restrict__ evicted)
+decode_step_split_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *__restrict__ k_new,
+                         const T *__restrict__ v_new, T *__restrict__ out, int32_t *__restrict__ evicted)
 {
     constexpr int VEC = Elem<T>::kVec;
     constexpr int LPR = D / VEC;          // lanes per row
     constexpr int RPW = 32 / LPR;         // rows per warp-wide load
     constexpr int NW = NT / 32;
-    static_assert(LPR <= 32 && 32 % LPR == 0, "row must fit a warp");
+    static_assert(LPR <= 32 && 32 % LPR == 0 && D <= 128, "row must fit a warp");
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
 
     extern __shared__ float smem[];
     const int M = c.M;
-    float *w = smem;                       // [M+1] logits, then exp(logit - max)
-    float *part = w + ((M + 1 + 3) & ~3);  // [NW][D] partial outputs
-    float *red = part + NW * D;            // [NW] reduction scratch
+    const int per_max = (M + C - 1) / C;
+    float *w = smem;                             // [per_max+1] logits, then exp(logit - max)
+    float *part = w + ((per_max + 1 + 3) & ~3);  // [NW][D] partial outputs
+    float *red = part + NW * D;                  // [NW] reduction scratch
+    __shared__ SplitExchange xch;
     __shared__ unsigned long long red_key[NW];
+    __shared__ int red_slot[NW];
     __shared__ int s_target;
 
-    const int u = blockIdx.x;
+    const int u = blockIdx.x / C;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, rsel = lane / LPR;
-    const int cnt = c.count[u];
+    const int cnt = min(c.count[u], M);
     const int p = c.len[u];
+    // this CTA's slice of the resident slots; rank 0 also owns the new token (local index nloc)
+    const int per = (cnt + C - 1) / C;
+    const int s0 = min(cnt, rank * per), s1 = min(cnt, s0 + per);
+    const int nloc = s1 - s0;
+    const int nsoft = nloc + (rank == 0 ? 1 : 0);
 
     T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
     T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
@@ -87,15 +121,15 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
     float qf[VEC];
     Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
 
-    // ---- (i) logits against every resident key, and against the new key -------
-    const int ngroups = (cnt + RPW - 1) / RPW;
+    // ---- (i) logits of the slice, and (rank 0) of the new key ---------------------------------
+    const int ngroups = (nloc + RPW - 1) / RPW;
     for (int g = warp; g < ngroups; g += NW * kUnroll) {
         uint4 r[kUnroll];
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
             const int row = (g + x * NW) * RPW + rsel;
             r[x] = make_uint4(0, 0, 0, 0);
-            if (row < cnt) r[x] = ld_stream16(Ku + (size_t)row * D + sub * VEC);
+            if (row < nloc) r[x] = ld_stream16(Ku + (size_t)(s0 + row) * D + sub * VEC);
         }
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
@@ -107,10 +141,10 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
             for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            if (sub == 0 && row < cnt) w[row] = dot * c.scale;
+            if (sub == 0 && row < nloc) w[row] = dot * c.scale;
         }
     }
-    if (warp == 0) {
+    if (warp == 0 && rank == 0) {
         float kf[VEC];
         Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC), kf);
         float dot = 0.f;
@@ -118,24 +152,23 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
         for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
         for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        if (lane == 0) w[cnt] = dot * c.scale;
+        if (lane == 0) w[nloc] = dot * c.scale;
     }
     __syncthreads();
 
-    // ---- (ii) softmax over resident + self ------------------------------------
-    float m = -INFINITY;
-    for (int s = tid; s <= cnt; s += NT) m = fmaxf(m, w[s]);
-    m = block_max<NT>(m, red);
-    float l = 0.f;
-    for (int s = tid; s <= cnt; s += NT) {
-        const float e = expf(w[s] - m);
+    // ---- (ii) local softmax statistics ----------------------------------------------------------
+    float m_loc = -INFINITY;
+    for (int s = tid; s < nsoft; s += NT) m_loc = fmaxf(m_loc, w[s]);
+    m_loc = block_max<NT>(m_loc, red);
+    float l_loc = 0.f;
+    for (int s = tid; s < nsoft; s += NT) {
+        const float e = expf(w[s] - m_loc);
         w[s] = e;
-        l += e;
+        l_loc += e;
     }
-    l = block_sum<NT>(l, red);
-    const float e_self = w[cnt];
+    l_loc = block_sum<NT>(l_loc, red);
 
-    // ---- (iii) out = (sum_s e_s V[s] + e_self v_new) / l ------------------------
+    // ---- (iii) unnormalised partial output of the slice -----------------------------------------
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
@@ -145,12 +178,12 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
         for (int x = 0; x < kUnroll; ++x) {
             const int row = (g + x * NW) * RPW + rsel;
             r[x] = make_uint4(0, 0, 0, 0);
-            if (row < cnt) r[x] = ld_stream16(Vu + (size_t)row * D + sub * VEC);
+            if (row < nloc) r[x] = ld_stream16(Vu + (size_t)(s0 + row) * D + sub * VEC);
         }
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
             const int row = (g + x * NW) * RPW + rsel;
-            const float ws = row < cnt ? w[row] : 0.f;
+            const float ws = row < nloc ? w[row] : 0.f;
             float vf[VEC];
             Elem<T>::unpack(r[x], vf);
 #pragma unroll
@@ -169,62 +202,105 @@ decode_step_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *_
         float o = 0.f;
 #pragma unroll
         for (int x = 0; x < NW; ++x) o += part[x * D + tid];
-        o = fmaf(e_self, Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+        if (rank == 0) o = fmaf(w[nloc], Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+        xch.out[tid] = o;
+    }
+    if (tid == 0) { xch.m = m_loc; xch.l = l_loc; }
+    cluster.sync();
+
+    // ---- global softmax constants: every CTA reads every (max, sum) pair, in rank order ----------
+    float m = -INFINITY;
+    for (int r2 = 0; r2 < C; ++r2) m = fmaxf(m, cluster.map_shared_rank(&xch, r2)->m);
+    float l = 0.f;
+    for (int r2 = 0; r2 < C; ++r2) {
+        const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
+        l += x->l * expf(x->m - m);          // an empty slice has m = -inf, l = 0
+    }
+    if (rank == 0 && tid < D) {
+        float o = 0.f;
+        for (int r2 = 0; r2 < C; ++r2) {
+            const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
+            o = fmaf(x->out[tid], expf(x->m - m), o);
+        }
         out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
     }
 
-    // ---- (iv) S <- alpha*S + a ; (v) argmin over the non-recent slots ------------
+    // ---- (iv) S <- alpha*S + a for the slice ; local eviction candidate ---------------------------
     const bool full = cnt >= M;
     const int newest_evictable = p - c.R;     // candidates: position <= p - R
+    const float rescale = expf(m_loc - m);
     unsigned long long best = ~0ull;
     int best_slot = -1;
-    for (int s = tid; s < cnt; s += NT) {
-        const float a = w[s] / l;
-        const float sn = fmaf(alpha, Su[s], a);
-        Su[s] = sn;
-        const int ps = posu[s];
+    for (int s = tid; s < nloc; s += NT) {
+        const float a = w[s] * rescale / l;
+        const float sn = fmaf(alpha, Su[s0 + s], a);
+        Su[s0 + s] = sn;
+        const int ps = posu[s0 + s];
         if (full && ps <= newest_evictable) {
             // scores are >= 0, so their bit patterns order like the values
             const unsigned long long key =
                 ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
-            if (key < best) { best = key; best_slot = s; }
+            if (key < best) { best = key; best_slot = s0 + s; }
         }
     }
-    const float a_self = e_self / l;
-    const unsigned long long wbest = warp_min_u64(best);
-    if (lane == 0) red_key[warp] = wbest;
-    if (tid == 0) s_target = full ? -2 : cnt;
-    __syncthreads();
-    unsigned long long gbest = red_key[0];
-#pragma unroll
-    for (int x = 1; x < NW; ++x) gbest = red_key[x] < gbest ? red_key[x] : gbest;
-    if (full && best_slot >= 0 && best == gbest) {
-        // positions are distinct, so exactly one thread holds the minimum
-        const unsigned long long self_key =
-            ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
-        if (c.R > 0 || gbest < self_key) s_target = best_slot;
+    // positions are distinct, so the minimum key identifies its slot
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+        if (ob < best) { best = ob; best_slot = os; }
     }
+    if (lane == 0) { red_key[warp] = best; red_slot[warp] = best_slot; }
     __syncthreads();
-
-    // ---- in-place insertion of the new token --------------------------------------
-    const int target = s_target;
-    if (target >= 0) {
-        if (tid < LPR)
-            *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
-                *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
-        else if (tid < 2 * LPR)
-            *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
-                *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
-    }
     if (tid == 0) {
-        if (target >= 0) {
-            Su[target] = a_self;
-            posu[target] = p;
-        }
-        if (!full) c.count[u] = cnt + 1;
-        c.len[u] = p + 1;
-        evicted[u] = full ? target : -1;
+        unsigned long long gb = red_key[0];
+        int gs = red_slot[0];
+        for (int x = 1; x < NW; ++x)
+            if (red_key[x] < gb) { gb = red_key[x]; gs = red_slot[x]; }
+        xch.best = gb;
+        xch.best_slot = gs;
     }
+    cluster.sync();
+
+    // ---- (v) rank 0 picks the global minimum and inserts the new token in place -------------------
+    if (rank == 0) {
+        const float a_self = w[nloc] * rescale / l;
+        if (tid == 0) {
+            int target = full ? -2 : cnt;
+            if (full) {
+                unsigned long long gb = ~0ull;
+                int gs = -1;
+                for (int r2 = 0; r2 < C; ++r2) {
+                    const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
+                    if (x->best < gb) { gb = x->best; gs = x->best_slot; }
+                }
+                const unsigned long long self_key =
+                    ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
+                if (gs >= 0 && (c.R > 0 || gb < self_key)) target = gs;
+            }
+            s_target = target;
+        }
+        __syncthreads();
+        const int target = s_target;
+        if (target >= 0) {
+            if (tid < LPR)
+                *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
+                    *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
+            else if (tid < 2 * LPR)
+                *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
+                    *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
+        }
+        if (tid == 0) {
+            if (target >= 0) {
+                Su[target] = a_self;
+                posu[target] = p;
+            }
+            if (!full) c.count[u] = cnt + 1;
+            c.len[u] = p + 1;
+            evicted[u] = full ? target : -1;
+        }
+    }
+    // peers must stay resident until rank 0 has read their shared memory
+    cluster.sync();
 }
 
 
@@ -596,24 +672,37 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
 }
 
 template <typename T, int D>
-cudaError_t launch_typed(const CacheView &c, float alpha, const void *q, const void *k_new,
-                         const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, const void *q,
+                         const void *k_new, const void *v_new, void *out, int32_t *evicted,
+                         cudaStream_t s)
 {
     constexpr int NT = kDecodeThreads;
-    const size_t smem = (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 + (size_t)(NT / 32) * D * 4 +
-                        (NT / 32) * 4;
-    auto kern = decode_step_kernel<T, D, NT>;
+    const size_t per_max = ((size_t)c.M + cluster_size - 1) / cluster_size;
+    const size_t smem = ((per_max + 1 + 3) & ~(size_t)3) * 4 + (size_t)(NT / 32) * D * 4 + (NT / 32) * 4;
+    auto kern = decode_step_split_kernel<T, D, NT>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<c.U, NT, smem, s>>>(c, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
-                               static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)c.U * cluster_size);
+    cfg.blockDim = dim3(NT);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, c, alpha, static_cast<const T *>(q),
+                                             static_cast<const T *>(k_new), static_cast<const T *>(v_new),
+                                             static_cast<T *>(out), evicted);
     count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
-
 
 template <typename T, int D>
 cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const void *k_new,
@@ -625,18 +714,26 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     // takes its share of the SM's shared memory
     constexpr int ctas_per_sm = kStreamCtasPerSm;
     const size_t per_cta = (227 * 1024) / ctas_per_sm - 1024;
-    if (fixed + 3 * kChunkBytes > per_cta) return launch_typed<T, D>(c, alpha, q, k_new, v_new, out, evicted, s);
+    if (fixed + 3 * kChunkBytes > per_cta) return launch_split<T, D>(c, 1, alpha, q, k_new, v_new, out, evicted, s);
     int stages = (int)((per_cta - fixed) / kChunkBytes);
     if (stages > kMaxStreamStages) stages = kMaxStreamStages;
     const size_t smem = fixed + (size_t)stages * kChunkBytes;
     auto kern = decode_step_stream_kernel<T, D>;
     static int num_sms = 0;
-    static cudaError_t attr_err = cudaSuccess;
-    static size_t attr_smem = 0;
-    if (num_sms == 0 || smem > attr_smem) {
+    if (num_sms == 0) {
         int dev = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    // Few units with long caches would leave most SMs idle: split each unit over a cluster.
+    if (c.M >= kSplitMinBudget && c.U * 2 <= num_sms) {
+        int cs = 2;
+        while (cs < 8 && c.U * cs * 2 <= 2 * num_sms) cs *= 2;
+        return launch_split<T, D>(c, cs, alpha, q, k_new, v_new, out, evicted, s);
+    }
+    static cudaError_t attr_err = cudaSuccess;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
         attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         attr_smem = smem;
     }

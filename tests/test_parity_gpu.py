@@ -67,6 +67,11 @@ def test_shrunken_configs(name, kw, alphas):
     dict(n=130, budget=40, recent=7, steps=8, dtype="bf16", d=64),
     dict(n=130, budget=40, recent=7, steps=8, dtype="fp16", d=64),
     dict(n=257, budget=300, recent=100, steps=50, dtype="bf16", d=128),
+    # long caches with few units run the cluster split-K decode kernel
+    dict(n=700, budget=513, recent=200, steps=30),                       # fp32, d = 64, odd budget
+    dict(n=520, budget=512, recent=0, steps=20, dtype="fp16", d=128),    # all selective
+    dict(n=100, budget=600, recent=10, steps=12),                        # most slices start empty
+    dict(n=9, budget=1024, recent=1024, steps=6, dtype="bf16", d=128),   # fewer tokens than CTAs
 ])
 def test_edge_cases(kw):
     w = W["tiny_fp32"].scaled(**kw)
