@@ -212,7 +212,7 @@ class Cache:
         self.torch_dtype = {v: k for k, v in _DTYPE_CODE.items()}[p.dtype]
 
     def close(self):
-        if getattr(self, "handle", None):
+        if getattr(self, "handle", None) and lib is not None:   # lib is None at interpreter exit
             lib.a2sf_cache_destroy(self.handle)
             self.handle = None
 
