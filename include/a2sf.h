@@ -105,6 +105,25 @@ int a2sf_rescore(const a2sf_params *p, int32_t n,
                  const float *lse, float *scores, int32_t *kept_idx,
                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Per-head forgetting factors (the paper's Limitation section suggests a distinct factor per
+ * layer and head instead of one uniform value).  `alphas` is a DEVICE array [B][H] fp32, one
+ * factor per unit; p->alpha is ignored.  Values outside [0, 1] (or NaN) cannot be rejected on
+ * the host and are clamped into [0, 1] on the device.  Everything else as in a2sf_prefill /
+ * a2sf_rescore. */
+int a2sf_prefill_per_head(const a2sf_params *p, int32_t n,
+                          const void *q, const void *k, const void *v,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                          const float *alphas,
+                          void *out, float *scores, int32_t *kept_idx, float *lse_opt,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+int a2sf_rescore_per_head(const a2sf_params *p, int32_t n,
+                          const void *q, const void *k,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                          const float *lse, const float *alphas,
+                          float *scores, int32_t *kept_idx,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Same as a2sf_prefill with HOST buffers: q, k, v, out contiguous [B][H][n][d];
  * scores, kept_idx as above, all in host memory (pinned memory makes the copies
  * asynchronous).  Inputs are copied to the device workspace, results copied back,
@@ -191,6 +210,12 @@ int a2sf_cache_load(a2sf_cache *cache, int32_t n, const void *k, const void *v,
 int a2sf_decode_step(a2sf_cache *cache, float alpha,
                      const void *q, const void *k_new, const void *v_new,
                      void *out, int32_t *evicted_slot, void *cuda_stream);
+
+/* The same step with one forgetting factor per unit: `alphas` is a DEVICE array [B][H] fp32
+ * (clamped into [0, 1] on the device).  See a2sf_prefill_per_head. */
+int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas,
+                              const void *q, const void *k_new, const void *v_new,
+                              void *out, int32_t *evicted_slot, void *cuda_stream);
 
 /* The same step with HOST buffers (pinned for asynchronous copies): q, k_new, v_new
  * are copied into staging rows inside the cache, the step runs, out and

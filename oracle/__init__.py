@@ -178,17 +178,28 @@ class Cache:
     def step(self, q, k_new, v_new, alpha: float, force=None, nthreads: int = 1):
         """One generation step for all units.  q, k_new, v_new: [U, d].
         ``force`` [U] int32: slot to vacate instead of the rule's choice when the
-        cache is full (-3 = follow the rule).  Returns out [U,d], info [U,3]
+        cache is full (-3 = follow the rule).  ``alpha`` may be a scalar or one value per
+        unit.  Returns out [U,d], info [U,3]
         (vacated, rule's choice, rule's runner-up) and their scores [U,3]."""
         q, k_new, v_new = _f64(q), _f64(k_new), _f64(v_new)
         out = np.empty((self.U, self.d), dtype=np.float64)
         info = np.empty((self.U, 3), dtype=np.int32)
         sc2 = np.empty((self.U, 3), dtype=np.float64)
         f = None if force is None else np.ascontiguousarray(force, dtype=np.int32)
-        self.lib.a2sf_oracle_decode_step_batch(
-            _dp(self.K), _dp(self.V), _dp(self.S), _ip(self.pos), _ip(self.count), _ip(self.len),
-            _dp(q), _dp(k_new), _dp(v_new), self.U, self.d, self.scale, float(alpha),
-            self.M, self.R, _ip(f), _dp(out), _ip(info), _dp(sc2), int(nthreads))
+        if np.ndim(alpha) == 0:
+            self.lib.a2sf_oracle_decode_step_batch(
+                _dp(self.K), _dp(self.V), _dp(self.S), _ip(self.pos), _ip(self.count), _ip(self.len),
+                _dp(q), _dp(k_new), _dp(v_new), self.U, self.d, self.scale, float(alpha),
+                self.M, self.R, _ip(f), _dp(out), _ip(info), _dp(sc2), int(nthreads))
+        else:
+            # one forgetting factor per unit: the single-unit step, unit by unit
+            assert len(alpha) == self.U
+            for u in range(self.U):
+                self.lib.a2sf_oracle_decode_step(
+                    _dp(self.K[u]), _dp(self.V[u]), _dp(self.S[u]), _ip(self.pos[u]),
+                    _ip(self.count[u:u + 1]), _ip(self.len[u:u + 1]), _dp(q[u]), _dp(k_new[u]),
+                    _dp(v_new[u]), self.d, self.scale, float(alpha[u]), self.M, self.R,
+                    -3 if f is None else int(f[u]), _dp(out[u]), _ip(info[u]), _dp(sc2[u]))
         return out, info, sc2
 
     def snapshot(self):

@@ -47,6 +47,9 @@ def _load():
     sigs = {
         "a2sf_prefill_workspace_bytes": (sz, [pp, i32]),
         "a2sf_prefill": (ctypes.c_int, [pp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]),
+        "a2sf_prefill_per_head": (ctypes.c_int, [pp, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, vp, sz, vp]),
+        "a2sf_rescore_per_head": (ctypes.c_int, [pp, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, vp, sz, vp]),
+        "a2sf_decode_step_per_head": (ctypes.c_int, [vp, vp, vp, vp, vp, vp, vp, vp]),
         "a2sf_rescore_workspace_bytes": (sz, [pp, i32]),
         "a2sf_rescore": (ctypes.c_int, [pp, i32, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]),
         "a2sf_prefill_static_scratch_max_rows": (sz, []),
@@ -125,8 +128,9 @@ def _strides(t: torch.Tensor):
 
 
 def a2sf_prefill(p: a2sf_params, q, k, v, out=None, scores=None, kept_idx=None, lse=None,
-                 workspace=None, stream=None):
-    """q, k, v: device [B,H,n,d].  Returns (out, scores, kept_idx, lse)."""
+                 workspace=None, stream=None, alphas=None):
+    """q, k, v: device [B,H,n,d].  Returns (out, scores, kept_idx, lse).
+    ``alphas``: optional device tensor [B,H] fp32 of per-head forgetting factors."""
     B, H, n, d = q.shape
     assert k.shape == q.shape and v.shape == q.shape
     assert _strides(k) == _strides(q) and _strides(v) == _strides(q)
@@ -142,14 +146,21 @@ def a2sf_prefill(p: a2sf_params, q, k, v, out=None, scores=None, kept_idx=None, 
         need = a2sf_prefill_workspace_bytes(p, n)
         workspace = torch.empty((max(need, 256),), dtype=torch.uint8, device=dev)
     sb, sh, st = _strides(q)
-    _check(lib.a2sf_prefill(ctypes.byref(p), n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st, _ptr(out),
-                            _ptr(scores), _ptr(kept_idx), _ptr(lse), _ptr(workspace),
-                            workspace.numel(), _stream(stream)), "a2sf_prefill")
+    if alphas is None:
+        _check(lib.a2sf_prefill(ctypes.byref(p), n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st, _ptr(out),
+                                _ptr(scores), _ptr(kept_idx), _ptr(lse), _ptr(workspace),
+                                workspace.numel(), _stream(stream)), "a2sf_prefill")
+    else:
+        assert alphas.dtype == torch.float32 and alphas.is_contiguous() and alphas.numel() == B * H
+        _check(lib.a2sf_prefill_per_head(ctypes.byref(p), n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st,
+                                         _ptr(alphas), _ptr(out), _ptr(scores), _ptr(kept_idx), _ptr(lse),
+                                         _ptr(workspace), workspace.numel(), _stream(stream)),
+               "a2sf_prefill_per_head")
     return out, scores, kept_idx, lse
 
 
 def a2sf_rescore(p: a2sf_params, q, k, lse, scores=None, kept_idx=None, workspace=None,
-                 stream=None):
+                 stream=None, alphas=None):
     """Scores and kept set for ``p.alpha`` from an existing log-sum-exp."""
     B, H, n, d = q.shape
     dev = q.device
@@ -161,10 +172,16 @@ def a2sf_rescore(p: a2sf_params, q, k, lse, scores=None, kept_idx=None, workspac
     if workspace is None:
         need = a2sf_rescore_workspace_bytes(p, n)
         workspace = torch.empty((need,), dtype=torch.uint8, device=dev) if need else None
-    _check(lib.a2sf_rescore(ctypes.byref(p), n, _ptr(q), _ptr(k), sb, sh, st, _ptr(lse),
-                            _ptr(scores), _ptr(kept_idx), _ptr(workspace),
-                            workspace.numel() if workspace is not None else 0,
-                            _stream(stream)), "a2sf_rescore")
+    wsn = workspace.numel() if workspace is not None else 0
+    if alphas is None:
+        _check(lib.a2sf_rescore(ctypes.byref(p), n, _ptr(q), _ptr(k), sb, sh, st, _ptr(lse),
+                                _ptr(scores), _ptr(kept_idx), _ptr(workspace), wsn,
+                                _stream(stream)), "a2sf_rescore")
+    else:
+        assert alphas.dtype == torch.float32 and alphas.is_contiguous() and alphas.numel() == B * H
+        _check(lib.a2sf_rescore_per_head(ctypes.byref(p), n, _ptr(q), _ptr(k), sb, sh, st, _ptr(lse),
+                                         _ptr(alphas), _ptr(scores), _ptr(kept_idx), _ptr(workspace), wsn,
+                                         _stream(stream)), "a2sf_rescore_per_head")
     return scores, kept_idx
 
 
@@ -230,6 +247,13 @@ class Cache:
     def a2sf_decode_step(self, alpha, q, k_new, v_new, out, evicted, stream=None):
         _check(lib.a2sf_decode_step(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),
                                     _ptr(out), _ptr(evicted), _stream(stream)), "a2sf_decode_step")
+
+    def a2sf_decode_step_per_head(self, alphas, q, k_new, v_new, out, evicted, stream=None):
+        """``alphas``: device tensor [B,H] fp32, one forgetting factor per unit."""
+        assert alphas.dtype == torch.float32 and alphas.is_contiguous() and alphas.numel() == self.U
+        _check(lib.a2sf_decode_step_per_head(self.handle, _ptr(alphas), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                             _ptr(out), _ptr(evicted), _stream(stream)),
+               "a2sf_decode_step_per_head")
 
     def a2sf_decode_step_host(self, alpha, q, k_new, v_new, out, evicted, stream=None):
         _check(lib.a2sf_decode_step_host(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),

@@ -89,10 +89,10 @@ size_t a2sf_rescore_workspace_bytes(const a2sf_params *p, int32_t n)
     return 0;
 }
 
-int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
-                 int64_t stride_b, int64_t stride_h, int64_t stride_t, void *out, float *scores,
-                 int32_t *kept_idx, float *lse_opt, void *workspace, size_t workspace_bytes,
-                 void *cuda_stream)
+static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
+                        int64_t stride_b, int64_t stride_h, int64_t stride_t, const float *alpha_vec,
+                        void *out, float *scores, int32_t *kept_idx, float *lse_opt, void *workspace,
+                        size_t workspace_bytes, void *cuda_stream)
 {
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
@@ -111,16 +111,36 @@ int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, 
     a.scores = scores;
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
-    a.scale = eff_scale(p); a.alpha = p->alpha;
+    a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     const cudaError_t e1 = prefill_tc_supported(p->dtype, a) ? launch_prefill_pass1_tc(p->dtype, a, s)
                                                              : launch_prefill_pass1_simt(p->dtype, a, s);
     if (e1 != cudaSuccess) return A2SF_ERR_CUDA;
     return run_scores_and_select(p, n, a, kept_idx, s);
 }
 
-int a2sf_rescore(const a2sf_params *p, int32_t n, const void *q, const void *k, int64_t stride_b,
-                 int64_t stride_h, int64_t stride_t, const float *lse, float *scores,
-                 int32_t *kept_idx, void *workspace, size_t workspace_bytes, void *cuda_stream)
+int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
+                 int64_t stride_b, int64_t stride_h, int64_t stride_t, void *out, float *scores,
+                 int32_t *kept_idx, float *lse_opt, void *workspace, size_t workspace_bytes,
+                 void *cuda_stream)
+{
+    return prefill_impl(p, n, q, k, v, stride_b, stride_h, stride_t, nullptr, out, scores, kept_idx,
+                        lse_opt, workspace, workspace_bytes, cuda_stream);
+}
+
+int a2sf_prefill_per_head(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t, const float *alphas,
+                          void *out, float *scores, int32_t *kept_idx, float *lse_opt,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!alphas || !aligned(alphas, 4)) return A2SF_ERR_INVALID_ARG;
+    return prefill_impl(p, n, q, k, v, stride_b, stride_h, stride_t, alphas, out, scores, kept_idx,
+                        lse_opt, workspace, workspace_bytes, cuda_stream);
+}
+
+static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const void *k, int64_t stride_b,
+                        int64_t stride_h, int64_t stride_t, const float *lse, const float *alpha_vec,
+                        float *scores, int32_t *kept_idx, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream)
 {
     (void)workspace; (void)workspace_bytes;
     int rc = check_params(p);
@@ -134,8 +154,26 @@ int a2sf_rescore(const a2sf_params *p, int32_t n, const void *q, const void *k, 
     a.scores = scores;
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
-    a.scale = eff_scale(p); a.alpha = p->alpha;
+    a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     return run_scores_and_select(p, n, a, kept_idx, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int a2sf_rescore(const a2sf_params *p, int32_t n, const void *q, const void *k, int64_t stride_b,
+                 int64_t stride_h, int64_t stride_t, const float *lse, float *scores,
+                 int32_t *kept_idx, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    return rescore_impl(p, n, q, k, stride_b, stride_h, stride_t, lse, nullptr, scores, kept_idx,
+                        workspace, workspace_bytes, cuda_stream);
+}
+
+int a2sf_rescore_per_head(const a2sf_params *p, int32_t n, const void *q, const void *k,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t, const float *lse,
+                          const float *alphas, float *scores, int32_t *kept_idx, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream)
+{
+    if (!alphas || !aligned(alphas, 4)) return A2SF_ERR_INVALID_ARG;
+    return rescore_impl(p, n, q, k, stride_b, stride_h, stride_t, lse, alphas, scores, kept_idx,
+                        workspace, workspace_bytes, cuda_stream);
 }
 
 size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n)
@@ -296,7 +334,22 @@ int a2sf_decode_step(a2sf_cache *cache, float alpha, const void *q, const void *
     if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16))
         return A2SF_ERR_INVALID_ARG;
-    if (launch_decode_step(cache->view, alpha, q, k_new, v_new, out, evicted_slot,
+    if (launch_decode_step(cache->view, alpha, nullptr, q, k_new, v_new, out, evicted_slot,
+                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas, const void *q,
+                              const void *k_new, const void *v_new, void *out,
+                              int32_t *evicted_slot, void *cuda_stream)
+{
+    if (!cache || !alphas || !q || !k_new || !v_new || !out || !evicted_slot)
+        return A2SF_ERR_INVALID_ARG;
+    if (!aligned(alphas, 4) || !aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) ||
+        !aligned(out, 16))
+        return A2SF_ERR_INVALID_ARG;
+    if (launch_decode_step(cache->view, cache->p.alpha, alphas, q, k_new, v_new, out, evicted_slot,
                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return A2SF_ERR_CUDA;
     return A2SF_OK;

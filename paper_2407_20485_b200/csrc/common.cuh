@@ -105,6 +105,7 @@ struct PrefillArgs {
     Strides st;
     int B, H, n, d;
     float scale, alpha;
+    const float *alpha_vec;   // per-unit forgetting factors [U] on the device, or nullptr (use alpha)
 };
 
 cudaError_t launch_prefill_pass1_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
@@ -133,8 +134,16 @@ cudaError_t launch_cache_load(const CacheView &c, int H, int n, const void *k, c
                               Strides st, const float *scores, const int32_t *kept,
                               cudaStream_t s);
 
-cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
-                               const void *v_new, void *out, int32_t *evicted, cudaStream_t s);
+// alpha_vec: per-unit forgetting factors [U] on the device, or nullptr (use the scalar)
+cudaError_t launch_decode_step(const CacheView &c, float alpha, const float *alpha_vec, const void *q,
+                               const void *k_new, const void *v_new, void *out, int32_t *evicted,
+                               cudaStream_t s);
+
+// per-unit factors are clamped to [0, 1] on the device (they cannot be validated on the host)
+__device__ __forceinline__ float unit_alpha(const float *alpha_vec, int u, float alpha)
+{
+    return alpha_vec ? fminf(fmaxf(alpha_vec[u], 0.f), 1.f) : alpha;
+}
 
 int read_and_clear_decode_status(cudaStream_t s);
 

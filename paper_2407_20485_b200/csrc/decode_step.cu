@@ -78,7 +78,8 @@ struct SplitExchange {
 
 template <typename T, int D, int NT>
 __global__ void __launch_bounds__(NT)
-decode_step_split_kernel(CacheView c, float alpha, const T *__restrict__ q, const T *__restrict__ k_new,
+decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__ alpha_vec,
+                         const T *__restrict__ q, const T *__restrict__ k_new,
                          const T *__restrict__ v_new, T *__restrict__ out, int32_t *__restrict__ evicted)
 {
     constexpr int VEC = Elem<T>::kVec;
@@ -103,6 +104,7 @@ decode_step_split_kernel(CacheView c, float alpha, const T *__restrict__ q, cons
     __shared__ int s_target;
 
     const int u = blockIdx.x / C;
+    const float alpha = unit_alpha(alpha_vec, u, alpha_all);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, rsel = lane / LPR;
     const int cnt = min(c.count[u], M);
@@ -386,7 +388,8 @@ struct StreamShared {
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kStreamThreads, 3)
-decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
+decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict__ alpha_vec,
+                          const T *__restrict__ q,
                           const T *__restrict__ k_new, const T *__restrict__ v_new,
                           T *__restrict__ out, int32_t *__restrict__ evicted, int *status,
                           int kStreamStages)
@@ -486,6 +489,7 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
             if (consumer_any(!got) || u < 0) break;        // uniform over the consumers
             if (lane == 0) tc::mbar_arrive(&sh->uq_empty[qi]);
             const int p = c.len[u];
+            const float alpha = unit_alpha(alpha_vec, u, alpha_all);
             T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
             T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
             float *Su = c.S + (size_t)u * M;
@@ -672,8 +676,8 @@ decode_step_stream_kernel(CacheView c, float alpha, const T *__restrict__ q,
 }
 
 template <typename T, int D>
-cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, const void *q,
-                         const void *k_new, const void *v_new, void *out, int32_t *evicted,
+cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, const float *alpha_vec,
+                         const void *q, const void *k_new, const void *v_new, void *out, int32_t *evicted,
                          cudaStream_t s)
 {
     constexpr int NT = kDecodeThreads;
@@ -697,7 +701,7 @@ cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, cons
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, c, alpha, static_cast<const T *>(q),
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, c, alpha, alpha_vec, static_cast<const T *>(q),
                                              static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                              static_cast<T *>(out), evicted);
     count_launch();
@@ -705,8 +709,8 @@ cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, cons
 }
 
 template <typename T, int D>
-cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const void *k_new,
-                          const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+cudaError_t launch_stream(const CacheView &c, float alpha, const float *alpha_vec, const void *q,
+                          const void *k_new, const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
     const size_t fixed = 128 + (((size_t)c.M + 1 + 3) & ~(size_t)3) * 4 +
                          (size_t)kStreamConsumerWarps * D * 4 + sizeof(StreamShared);
@@ -714,7 +718,7 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     // takes its share of the SM's shared memory
     constexpr int ctas_per_sm = kStreamCtasPerSm;
     const size_t per_cta = (227 * 1024) / ctas_per_sm - 1024;
-    if (fixed + 3 * kChunkBytes > per_cta) return launch_split<T, D>(c, 1, alpha, q, k_new, v_new, out, evicted, s);
+    if (fixed + 3 * kChunkBytes > per_cta) return launch_split<T, D>(c, 1, alpha, alpha_vec, q, k_new, v_new, out, evicted, s);
     int stages = (int)((per_cta - fixed) / kChunkBytes);
     if (stages > kMaxStreamStages) stages = kMaxStreamStages;
     const size_t smem = fixed + (size_t)stages * kChunkBytes;
@@ -729,7 +733,7 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     if (c.M >= kSplitMinBudget && c.U * 2 <= num_sms) {
         int cs = 2;
         while (cs < 8 && c.U * cs * 2 <= 2 * num_sms) cs *= 2;
-        return launch_split<T, D>(c, cs, alpha, q, k_new, v_new, out, evicted, s);
+        return launch_split<T, D>(c, cs, alpha, alpha_vec, q, k_new, v_new, out, evicted, s);
     }
     static cudaError_t attr_err = cudaSuccess;
     static size_t attr_smem = 0;
@@ -741,7 +745,7 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
     int *status = decode_status_word();
     if (!status) return cudaErrorUnknown;
     const int grid = c.U < ctas_per_sm * num_sms ? c.U : ctas_per_sm * num_sms;
-    kern<<<grid, kStreamThreads, smem, s>>>(c, alpha, static_cast<const T *>(q),
+    kern<<<grid, kStreamThreads, smem, s>>>(c, alpha, alpha_vec, static_cast<const T *>(q),
                                             static_cast<const T *>(k_new), static_cast<const T *>(v_new),
                                             static_cast<T *>(out), evicted, status, stages);
     count_launch();
@@ -750,12 +754,13 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const void *q, const 
 
 }  // namespace
 
-cudaError_t launch_decode_step(const CacheView &c, float alpha, const void *q, const void *k_new,
-                               const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+cudaError_t launch_decode_step(const CacheView &c, float alpha, const float *alpha_vec, const void *q,
+                               const void *k_new, const void *v_new, void *out, int32_t *evicted,
+                               cudaStream_t s)
 {
 #define A2SF_DISPATCH(T)                                                                     \
-    (c.d == 64 ? launch_stream<T, 64>(c, alpha, q, k_new, v_new, out, evicted, s)            \
-               : launch_stream<T, 128>(c, alpha, q, k_new, v_new, out, evicted, s))
+    (c.d == 64 ? launch_stream<T, 64>(c, alpha, alpha_vec, q, k_new, v_new, out, evicted, s)  \
+               : launch_stream<T, 128>(c, alpha, alpha_vec, q, k_new, v_new, out, evicted, s))
     switch (c.dtype) {
     case A2SF_F32: return A2SF_DISPATCH(float);
     case A2SF_BF16: return A2SF_DISPATCH(__nv_bfloat16);

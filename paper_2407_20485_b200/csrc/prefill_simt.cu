@@ -166,7 +166,8 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
 
     // weight alpha^(n-1-i) folded into the exponent: exp2(s*log2e - c_i),
     // c_i = lse_i*log2e - (n-1-i)*log2(alpha); alpha = 0 keeps only row n-1 (0^0 = 1).
-    const float neg_log2_alpha = a.alpha > 0.f ? -log2f(a.alpha) : INFINITY;
+    const float alpha = unit_alpha(a.alpha_vec, u, a.alpha);
+    const float neg_log2_alpha = alpha > 0.f ? -log2f(alpha) : INFINITY;
     const float sl2 = a.scale * kLog2e;
 
     float acc = 0.f;

@@ -82,6 +82,7 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
     a.alpha = p->alpha;
+    a.alpha_vec = nullptr;
     if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
     if (launch_prefill_pass2_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
     if (launch_select(scores, kept_idx, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)

@@ -38,7 +38,8 @@ struct ScoreArgs {
     float *scores;        // [U][n]
     int n, H;
     float sl2;            // scale * log2(e)
-    float neg_log2_alpha; // -log2(alpha); +inf for alpha = 0
+    float alpha;          // forgetting factor, or per unit:
+    const float *alpha_vec;
 };
 
 struct ScoreShared {
@@ -180,6 +181,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         const int j = kb * kBlk + key_lane;
         const int et = threadIdx.x - 64;            // 0..255
         const float *lse = a.lse + (size_t)u * a.n;
+        const float alpha = unit_alpha(a.alpha_vec, u, a.alpha);
+        const float neg_log2_alpha = alpha > 0.f ? -log2f(alpha) : INFINITY;   // alpha = 0: only row n-1
         // A failed wait poisons the CTA: later waits return at once and the loop keeps its
         // shape, so every thread still reaches the final barrier; the status word reports it.
         auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
@@ -192,7 +195,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         auto row_const = [&](int i) -> float {
             if (i >= a.n) return INFINITY;
             const int age = a.n - 1 - i;
-            return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * a.neg_log2_alpha);
+            return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha);
         };
         float c_next = hsel == 0 ? row_const(kb * kBlk + et) : 0.f;
         float sum = 0.f;
@@ -709,7 +712,8 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     ScoreArgs sa;
     sa.lse = a.lse; sa.scores = a.scores; sa.n = a.n; sa.H = a.H;
     sa.sl2 = a.scale * kLog2e;
-    sa.neg_log2_alpha = a.alpha > 0.f ? -log2f(a.alpha) : INFINITY;
+    sa.alpha = a.alpha;
+    sa.alpha_vec = a.alpha_vec;
     const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
     score_pass_tc<<<grid, kScoreThreads, kScoreSmemBytes, s>>>(mq, mk, sa, dtype == A2SF_BF16 ? 1 : 0);
     count_launch();

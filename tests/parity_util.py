@@ -95,12 +95,14 @@ def make_inputs(w: wl.Workload, device, steps: int):
 def run_parity(w: wl.Workload, device="cuda", units: Optional[Sequence[int]] = None,
                alphas: Optional[Sequence[float]] = None, steps: Optional[int] = None,
                nthreads: Optional[int] = None, check_every: int = 1,
-               inputs=None) -> ParityReport:
+               inputs=None, alpha_units=None) -> ParityReport:
     """Prefill + cache build + ``steps`` decode steps on the GPU for ALL units of
     ``w``; the oracle follows the units listed in ``units`` (default: all).
 
     ``alphas``: extra forgetting factors whose scores / kept sets are checked through
-    ``a2sf_rescore`` (the decode phase always uses ``w.alpha``)."""
+    ``a2sf_rescore`` (the decode phase always uses ``w.alpha``).
+    ``alpha_units``: float32 array [w.units], one forgetting factor per (batch, head): the
+    per-head entry points are used and the oracle runs every unit with its own factor."""
     rep = ParityReport()
     nthreads = nthreads or oracle.host_threads()
     T = w.steps if steps is None else steps
@@ -122,11 +124,25 @@ def run_parity(w: wl.Workload, device="cuda", units: Optional[Sequence[int]] = N
 
     # ---- prefill -------------------------------------------------------------------
     p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
-    out_g, S_g, kept_g, lse_g = a2sf.a2sf_prefill(p, q, k, v)
+    alphas_t = None
+    if alpha_units is not None:
+        alpha_units = np.asarray(alpha_units, dtype=np.float32)
+        assert alpha_units.shape == (w.units,) and not alphas
+        alphas_t = torch.from_numpy(alpha_units).view(w.B, w.H).to(device)
+    out_g, S_g, kept_g, lse_g = a2sf.a2sf_prefill(p, q, k, v, alphas=alphas_t)
     torch.cuda.synchronize()
     all_alphas = [w.alpha] + [a for a in (alphas or []) if a != w.alpha]
-    ref = oracle.prefill(Qo, Ko, Vo, w.scale, all_alphas, w.budget, w.recent, sel_alpha=0,
-                         nthreads=nthreads)
+    if alpha_units is None:
+        ref = oracle.prefill(Qo, Ko, Vo, w.scale, all_alphas, w.budget, w.recent, sel_alpha=0,
+                             nthreads=nthreads)
+    else:
+        per = [oracle.prefill(Qo[x:x + 1], Ko[x:x + 1], Vo[x:x + 1], w.scale, [float(alpha_units[uu])],
+                              w.budget, w.recent) for x, uu in enumerate(units)]
+        ref = {key: np.concatenate([r[key] for r in per]) for key in ("out", "lse", "S", "kept")}
+        # the second pass alone, from the saved log-sum-exp, must give the same scores
+        S2, kept2 = a2sf.a2sf_rescore(p, q, k, lse_g, alphas=alphas_t)
+        torch.cuda.synchronize()
+        assert torch.equal(S2, S_g) and torch.equal(kept2, kept_g)
     check_out(pick(out_g), ref["out"], w.dtype, rep, "prefill out")
     lse_err = np.abs(pick(lse_g) - ref["lse"]).max()
     assert lse_err <= 1e-4 * max(1.0, np.abs(ref["lse"]).max()), f"lse off by {lse_err}"
@@ -174,11 +190,15 @@ def run_parity(w: wl.Workload, device="cuda", units: Optional[Sequence[int]] = N
     out_t = torch.empty((w.B, w.H, w.d), dtype=w.torch_dtype, device=device)
     ev_t = torch.empty((w.B, w.H), dtype=torch.int32, device=device)
     for t in range(T):
-        cache.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], out_t, ev_t)
+        if alphas_t is None:
+            cache.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], out_t, ev_t)
+        else:
+            cache.a2sf_decode_step_per_head(alphas_t, dq[t], dk[t], dv[t], out_t, ev_t)
         torch.cuda.synchronize()
         ev_g = pick_i(ev_t).astype(np.int32)
         force = np.where(ev_g == -1, -3, ev_g).astype(np.int32)
-        o_out, info, sc = ocache.step(pick(dq[t]), pick(dk[t]), pick(dv[t]), w.alpha, force=force,
+        step_alpha = w.alpha if alpha_units is None else [float(alpha_units[uu]) for uu in units]
+        o_out, info, sc = ocache.step(pick(dq[t]), pick(dk[t]), pick(dv[t]), step_alpha, force=force,
                                       nthreads=nthreads)
         for x in range(len(units)):
             if info[x, 1] == -1:

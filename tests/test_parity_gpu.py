@@ -168,6 +168,30 @@ def test_export_import_round_trip_and_generator_on_device():
     assert a2sf.a2sf_kernel_launch_count() > 0
 
 
+# ---- one forgetting factor per head (the paper's Limitation section) -------------------------
+@pytest.mark.parametrize("name,kw", [
+    ("llama2_7b", dict(B=2, H=3, n=500, steps=30)),              # tensor-core prefill, streaming decode
+    ("tiny_fp32", dict(H=5, n=150, steps=20)),                   # CUDA-core prefill
+    ("long_context", dict(H=2, n=1300, budget=600, recent=100, steps=16)),   # split-K decode
+])
+def test_per_head_forgetting_factors(name, kw):
+    from parity_util import run_parity
+
+    w = W[name].scaled(**kw)
+    alphas = np.array([0.0, 0.1, 0.3, 0.5, 0.9, 1.0], dtype=np.float32)[np.arange(w.units) % 6]
+    rep = run_parity(w, alpha_units=alphas)
+    assert rep.decode_evictions == w.units * w.steps
+    # a different factor per head must matter: the uniform run gives different scores
+    from paper_2407_20485_b200 import binding as a2sf
+    q, k, v = (t.cuda() for t in wl.make_prompt(w))
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, 0.5)
+    _, S_uniform, _, _ = a2sf.a2sf_prefill(p, q, k, v)
+    _, S_heads, _, _ = a2sf.a2sf_prefill(p, q, k, v, alphas=torch.from_numpy(alphas).view(w.B, w.H).cuda())
+    torch.cuda.synchronize()
+    same = [torch.equal(S_uniform.view(w.units, -1)[u], S_heads.view(w.units, -1)[u]) for u in range(w.units)]
+    assert same == [bool(a == 0.5) for a in alphas]
+
+
 # ---- the stated configurations at full size, oracle on sampled units ------------------
 @pytest.mark.parametrize("name,n_units,steps", [
     ("llama2_7b", 32, 256),
