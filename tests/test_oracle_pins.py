@@ -386,3 +386,29 @@ def test_batch_threads_do_not_change_results():
         np.testing.assert_array_equal(a[key], b[key])
     for u in range(U):
         np.testing.assert_array_equal(a["kept"][u], oracle.select(a["S"][u, 1], 8, 4))
+
+
+def test_per_unit_alpha_equals_unit_by_unit_scalar_steps():
+    """A vector of forgetting factors is the scalar step applied unit by unit."""
+    rng = np.random.default_rng(14)
+    U, d, M, R = 3, 8, 6, 2
+    K, V = rng.standard_normal((2, U, M, d))
+    S = rng.random((U, M))
+    kept = np.tile(np.arange(M, dtype=np.int32), (U, 1))
+    alphas = [0.0, 0.4, 1.0]
+    a = oracle.Cache(U, d, M, R, 0.3)
+    a.load(K, V, S, kept)
+    singles = []
+    for u in range(U):
+        c = oracle.Cache(1, d, M, R, 0.3)
+        c.load(K[u:u + 1], V[u:u + 1], S[u:u + 1], kept[u:u + 1])
+        singles.append(c)
+    for t in range(5):
+        q, k, v = rng.standard_normal((3, U, d))
+        out, info, sc = a.step(q, k, v, alphas)
+        for u in range(U):
+            o1, i1, s1 = singles[u].step(q[u:u + 1], k[u:u + 1], v[u:u + 1], alphas[u])
+            np.testing.assert_array_equal(out[u], o1[0])
+            np.testing.assert_array_equal(info[u], i1[0])
+            np.testing.assert_array_equal(a.S[u], singles[u].S[0])
+            np.testing.assert_array_equal(a.pos[u], singles[u].pos[0])
