@@ -50,7 +50,7 @@ def load_peaks():
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
 
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    FIELDS = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -79,7 +79,11 @@ class ClockSampler:
             except subprocess.TimeoutExpired:
                 self.proc.kill()
 
-    def summary(self):
+    def summary(self, t0=None, t1=None):
+        """Median SM clock and throttle reasons of the samples taken between the wall-clock
+        instants t0 and t1 (datetime, local time; None = no bound)."""
+        from datetime import datetime
+
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if not self.path or not os.path.exists(self.path):
             return out
@@ -87,14 +91,18 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             parts = [x.strip() for x in line.split(",")]
-            if len(parts) < 9:
+            if len(parts) < 10:
                 continue
             try:
-                sm.append(float(parts[1]))
-                mx.append(float(parts[2]))
+                ts = datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f")
+                if (t0 and ts < t0) or (t1 and ts > t1):
+                    continue
+                sm_v, mx_v = float(parts[2]), float(parts[3])
             except ValueError:
                 continue
-            for name, val in zip(names, parts[5:9]):
+            sm.append(sm_v)
+            mx.append(mx_v)
+            for name, val in zip(names, parts[6:10]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         os.unlink(self.path)
@@ -147,21 +155,26 @@ def run_ours(args):
             cache.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o_t[t], e_t[t])
         if ev: ev[3].record()
 
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    a2dist.barrier()
-    evs = [cuda_events(4) for _ in range(args.steps)]
-    launches0 = a2sf.a2sf_kernel_launch_count()
+    from datetime import datetime
+
+    # the sampler starts before the warm-up (nvidia-smi needs a moment to come up); only the
+    # samples that fall inside the timed region are reported
     with ClockSampler(local_rank) as clk:
+        for _ in range(args.warmup):
+            step()
         torch.cuda.synchronize()
+        a2dist.barrier()
+        evs = [cuda_events(4) for _ in range(args.steps)]
+        launches0 = a2sf.a2sf_kernel_launch_count()
         t_start = cuda_events(1)[0]
         t_end = cuda_events(1)[0]
+        wall0 = datetime.now()
         t_start.record()
         for i in range(args.steps):
             step(evs[i])
         t_end.record()
         torch.cuda.synchronize()
+        wall1 = datetime.now()
     a2dist.barrier()
     launches = a2sf.a2sf_kernel_launch_count() - launches0
     assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
@@ -169,7 +182,7 @@ def run_ours(args):
     prefill_ms = sum(e[0].elapsed_time(e[1]) for e in evs)
     load_ms = sum(e[1].elapsed_time(e[2]) for e in evs)
     decode_ms = sum(e[2].elapsed_time(e[3]) for e in evs)
-    clocks = clk.summary()
+    clocks = clk.summary(wall0, wall1)
 
     # ---- end to end through the host-buffer entry points (copies inside the timed region)
     e2e = None
@@ -364,7 +377,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2_13b", choices=sorted(wl.WORKLOADS))
