@@ -46,7 +46,8 @@ static int check_strides(const a2sf_params *p, int64_t sb, int64_t sh, int64_t s
 // prefill workspace: the log-sum-exp rows when the caller does not keep them
 static size_t prefill_ws_bytes(const a2sf_params *p, int n)
 {
-    return align_up((size_t)p->B * p->H * n * sizeof(float));
+    return align_up((size_t)p->B * p->H * n * sizeof(float)) +
+           prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d);
 }
 
 static int run_scores_and_select(const a2sf_params *p, int n, PrefillArgs &a, int32_t *kept,
@@ -112,6 +113,12 @@ static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
+    a.v_half = nullptr; a.v_flag = nullptr;
+    if (prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d) > 0) {
+        char *extra = static_cast<char *>(workspace) + align_up((size_t)p->B * p->H * n * sizeof(float));
+        a.v_flag = reinterpret_cast<int *>(extra);
+        a.v_half = extra + 256;
+    }
     const cudaError_t e1 = prefill_tc_supported(p->dtype, a) ? launch_prefill_pass1_tc(p->dtype, a, s)
                                                              : launch_prefill_pass1_simt(p->dtype, a, s);
     if (e1 != cudaSuccess) return A2SF_ERR_CUDA;
@@ -155,6 +162,7 @@ static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
+    a.v_half = nullptr; a.v_flag = nullptr;
     return run_scores_and_select(p, n, a, kept_idx, static_cast<cudaStream_t>(cuda_stream));
 }
 

@@ -106,6 +106,8 @@ struct PrefillArgs {
     int B, H, n, d;
     float scale, alpha;
     const float *alpha_vec;   // per-unit forgetting factors [U] on the device, or nullptr (use alpha)
+    void *v_half;             // bf16 tensor-core path: fp16 copy of V, contiguous [U][n][d] (workspace)
+    int *v_flag;              // ... and the word that says the copy is not exact (workspace)
 };
 
 cudaError_t launch_prefill_pass1_simt(int dtype, const PrefillArgs &a, cudaStream_t s);
@@ -113,6 +115,8 @@ cudaError_t launch_prefill_pass2_simt(int dtype, const PrefillArgs &a, cudaStrea
 
 // tensor-core path (16-bit storage, d = 128)
 bool prefill_tc_supported(int dtype, const PrefillArgs &a);
+// extra workspace of the tensor-core attention pass (fp16 copy of V + flag; bf16 storage only)
+size_t prefill_tc_extra_bytes(int dtype, size_t units, int n, int d);
 cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 int read_and_clear_tc_status(cudaStream_t s);

@@ -10,6 +10,7 @@
 // owner, warps 2-9 = epilogue.  A key is shared by two threads, one per 64-row half of the
 // query tile (more warps per scheduler keep the special-function unit fed); each keeps its
 // own running sum in row order and the two are added once at the end, in a fixed order.
+#include <algorithm>
 #include <mutex>
 #include <type_traits>
 
@@ -286,6 +287,8 @@ struct AttnArgs {
     int64_t st_b, st_h, st_t;
     int n, H;
     float sl2;            // scale * log2(e)
+    const int *v_flag;    // bf16 storage: 0 = the fp16 copy of V is exact, 1 = it is not
+    int run_if_flag;      // this launch works only when *v_flag equals this value
 };
 
 struct AttnShared {
@@ -311,14 +314,22 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-template <typename T>
+// PvHalf (bf16 storage only): the P V product runs in fp16 -- P is rounded to fp16 (11
+// significand bits, one term) and V comes from an fp16 copy made beforehand.  The launch works
+// only if that copy is exact (*v_flag == 0); otherwise the plain bf16 launch, which writes P as
+// two bf16 terms, does the work.
+template <typename T, bool PvHalf>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
              const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
 {
     // once any CTA has given up on a wait, the rest of the grid drains without working
     __shared__ int s_skip;
-    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile int *>(&g_tc_status);
+    if (threadIdx.x == 0) {
+        int skip = *reinterpret_cast<volatile int *>(&g_tc_status);
+        if (a.v_flag && (*a.v_flag != 0) != (a.run_if_flag != 0)) skip = 1;   // the other launch's job
+        s_skip = skip;
+    }
     __syncthreads();
     if (s_skip) return;
 
@@ -331,11 +342,13 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     AttnShared *sh = reinterpret_cast<AttnShared *>(Vs + kVStages * kTileBytes);
 
     constexpr int ab_fmt = std::is_same<T, __nv_bfloat16>::value ? 1 : 0;
+    using PT = typename std::conditional<PvHalf, __half, T>::type;      // element type of P and V
+    constexpr int pv_fmt = std::is_same<PT, __nv_bfloat16>::value ? 1 : 0;
     // A bf16 probability keeps 8 significand bits; where the products p*v cancel, that
     // rounding alone exceeds the output tolerance.  For bf16 the probabilities are therefore
     // split into two bf16 terms (p = hi + lo, |lo| <= 2^-9 |hi|) and both are multiplied
     // with V.  fp16 keeps 11 bits and needs no second term.
-    constexpr bool kSplitP = std::is_same<T, __nv_bfloat16>::value;
+    constexpr bool kSplitP = std::is_same<PT, __nv_bfloat16>::value;
 
     // CTAs of one unit are adjacent in the grid (longest rows first), so they run together
     // and share the unit's K and V tiles through L2
@@ -419,7 +432,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         // ---- MMA issuer -----------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc_qk = make_idesc(ab_fmt, kBlk, kBlk, 0, 0);
-            const uint32_t idesc_pv = make_idesc(ab_fmt, kBlk, kD, 0, 1);     // V is MN-major
+            const uint32_t idesc_pv = make_idesc(pv_fmt, kBlk, kD, 0, 1);     // V is MN-major
             uint64_t q_desc[2], k_desc[kKStages], v_desc[kVStages];
             for (int x = 0; x < 2; ++x) q_desc[x] = kmajor_desc(smem_u32(Qs + x * kTileBytes));
             for (int x = 0; x < kKStages; ++x) k_desc[x] = kmajor_desc(smem_u32(Ks + x * kTileBytes));
@@ -555,9 +568,9 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                             if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
                         }
                         rowsum += p0 + p1;
-                        hi[e] = pack2<T>(p0, p1);
+                        hi[e] = pack2<PT>(p0, p1);
                         if (kSplitP)      // a bf16 is the upper half of an fp32
-                            lo[e] = pack2<T>(p0 - __uint_as_float(hi[e] << 16),
+                            lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
                                              p1 - __uint_as_float(hi[e] & 0xffff0000u));
                     }
                     tmem_st16(sp + c * 16, hi);
@@ -621,6 +634,37 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     if (threadIdx.x == 0 && sh->abort_flag) g_tc_status = A2SF_ERR_TIMEOUT;
 }
 
+// fp16 copy of a bf16 V tensor, contiguous [U][n][d], for the PvHalf attention launch.  A bf16
+// value converts exactly when its magnitude is within fp16's range (magnitudes below 2^-17 lose
+// at most 2^-25 absolutely, which is immaterial); any value beyond 65504, infinite or NaN raises
+// the flag, and the attention pass then multiplies in bf16.
+__global__ void v_to_half_kernel(const __nv_bfloat16 *__restrict__ v, Strides st, int H, int n,
+                                 size_t chunks, __half *__restrict__ dst, int *__restrict__ flag)
+{
+    constexpr int CH = kD / 8;                       // 16-byte chunks per row
+    int bad = 0;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < chunks;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % CH);
+        const size_t row = idx / CH;
+        const int t = (int)(row % n);
+        const size_t u = row / n;
+        const size_t b = u / H, h = u % H;
+        const uint4 raw = ld_stream16(v + b * st.b + h * st.h + (size_t)t * st.t + c * 8);
+        float f[8];
+        Elem<__nv_bfloat16>::unpack(raw, f);
+        uint4 o;
+        __half2 *oh = reinterpret_cast<__half2 *>(&o);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            bad |= !(fabsf(f[2 * e]) <= 65504.f) | !(fabsf(f[2 * e + 1]) <= 65504.f);   // also NaN
+            oh[e] = __floats2half2_rn(f[2 * e], f[2 * e + 1]);
+        }
+        *reinterpret_cast<uint4 *>(dst + idx * 8) = o;
+    }
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1);
+}
+
 // ---- host: tensor maps -----------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -643,12 +687,14 @@ EncodeTiledFn encode_fn()
 
 // [B][H][n][d] 16-bit tensor -> 4-D map (d, n, H, B), box 64 x 128 rows, 128-byte swizzle,
 // out-of-range rows read as zero.
-bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillArgs &a)
+bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillArgs &a,
+                   const Strides *override_strides = nullptr)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
+    const Strides st = override_strides ? *override_strides : a.st;
     const cuuint64_t dims[4] = {(cuuint64_t)a.d, (cuuint64_t)a.n, (cuuint64_t)a.H, (cuuint64_t)a.B};
-    const cuuint64_t strides[3] = {(cuuint64_t)a.st.t * 2, (cuuint64_t)a.st.h * 2, (cuuint64_t)a.st.b * 2};
+    const cuuint64_t strides[3] = {(cuuint64_t)st.t * 2, (cuuint64_t)st.h * 2, (cuuint64_t)st.b * 2};
     const cuuint32_t box[4] = {64, (cuuint32_t)kBlk, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     const CUtensorMapDataType dt =
@@ -666,6 +712,12 @@ bool prefill_tc_supported(int dtype, const PrefillArgs &a)
            (size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk) < 0x7fffffffull;
 }
 
+size_t prefill_tc_extra_bytes(int dtype, size_t units, int n, int d)
+{
+    if (dtype != A2SF_BF16 || d != kD) return 0;
+    return 256 + ((units * (size_t)n * d * 2 + 255) / 256) * 256;      // flag word + fp16 copy of V
+}
+
 cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
 {
     CUtensorMap mq, mk, mv;
@@ -675,11 +727,12 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+        const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+        attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, false>, attr, (int)kAttnSmemBytes);
         if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_pass_tc<__half>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+            attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, true>, attr, (int)kAttnSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(attn_pass_tc<__half, false>, attr, (int)kAttnSmemBytes);
     });
     if (attr_err != cudaSuccess) return attr_err;
     AttnArgs aa;
@@ -687,12 +740,39 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
     aa.n = a.n; aa.H = a.H;
     aa.sl2 = a.scale * kLog2e;
+    aa.v_flag = nullptr; aa.run_if_flag = 0;
     const int npairs = ((a.n + kBlk - 1) / kBlk + 1) / 2;
     const dim3 grid((unsigned)((size_t)a.B * a.H * npairs));
-    if (dtype == A2SF_BF16)
-        attn_pass_tc<__nv_bfloat16><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
-    else
-        attn_pass_tc<__half><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+    if (dtype == A2SF_F16) {
+        attn_pass_tc<__half, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+        count_launch();
+        return cudaGetLastError();
+    }
+    if (!a.v_half || !a.v_flag) {       // no room for the fp16 copy: multiply in bf16
+        attn_pass_tc<__nv_bfloat16, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+        count_launch();
+        return cudaGetLastError();
+    }
+    // bf16: make the fp16 copy of V, then launch both forms of the pass; the flag written by
+    // the copy decides on the device which of the two does the work (no host round trip)
+    cudaError_t e = cudaMemsetAsync(a.v_flag, 0, sizeof(int), s);
+    if (e != cudaSuccess) return e;
+    const size_t chunks = (size_t)a.B * a.H * a.n * (kD / 8);
+    const unsigned cgrid = (unsigned)std::min<size_t>((chunks + 255) / 256, 148 * 16);
+    v_to_half_kernel<<<cgrid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(a.v), a.st, a.H, a.n, chunks,
+                                           static_cast<__half *>(a.v_half), a.v_flag);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    const Strides contig{(int64_t)a.H * a.n * kD, (int64_t)a.n * kD, (int64_t)kD};
+    CUtensorMap mvh;
+    if (!make_tile_map(&mvh, A2SF_F16, a.v_half, a, &contig)) return cudaErrorInvalidValue;
+    aa.v_flag = a.v_flag;
+    aa.run_if_flag = 0;
+    attn_pass_tc<__nv_bfloat16, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mvh, aa);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    aa.run_if_flag = 1;
+    attn_pass_tc<__nv_bfloat16, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
     count_launch();
     return cudaGetLastError();
 }

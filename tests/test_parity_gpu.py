@@ -104,6 +104,22 @@ def test_strided_inputs_and_determinism():
     run_parity(w, inputs=(qs, ks, vs, None, None, None))
 
 
+def test_values_beyond_fp16_range_take_the_bf16_product():
+    """bf16 V is multiplied through an fp16 copy when that copy is exact; values above 65504
+    (or inf / NaN) must switch, on the device, to the two-term bf16 product."""
+    from parity_util import make_inputs, run_parity
+
+    w = W["llama2_7b"].scaled(H=2, n=500, steps=6)
+    q, k, v, dq, dk, dv = make_inputs(w, "cuda", w.steps)
+    big = (v.float() * 3.0e5).to(v.dtype)                    # |v| up to ~1e6: not representable in fp16
+    assert big.float().abs().max() > 65504
+    rep = run_parity(w, inputs=(q, k, big, dq, dk, (dv.float() * 3.0e5).to(dv.dtype)))
+    assert rep.max_out_err <= 1.0
+    one = v.clone()
+    one[0, 1, 7, 3] = 7.0e4                                  # a single element beyond the range
+    run_parity(w, inputs=(q, k, one, dq, dk, dv))
+
+
 def test_host_buffer_entry_points_match_device_ones():
     from paper_2407_20485_b200 import binding as a2sf
 
