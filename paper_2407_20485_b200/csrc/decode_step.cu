@@ -320,12 +320,24 @@ constexpr int kMaxStreamStages = 12;
 constexpr int kStreamCtasPerSm = 3;          // measured best on config 4 (2: 63.8 us, 3: 60.5 us, 4: 68.6 us)
 constexpr int kPrefetchSlots = 2;            // score/position words each consumer thread preloads
 
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar)
+// The cache is streamed once per step and never re-read before the next step, by which time
+// the rest of the cache has passed through L2: marking the copies evict-first keeps them from
+// displacing one another's lines in flight (measured on config 4: 61.0 -> 55.7 us per step).
+__device__ __forceinline__ uint64_t evict_first_policy()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar,
+                                          uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1], %2, [%3], %4;"
         :
-        : "r"(tc::smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(tc::smem_u32(bar))
+        : "r"(tc::smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(tc::smem_u32(bar)), "l"(policy)
         : "memory");
 }
 
@@ -434,6 +446,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             int stage = 0;
             uint32_t phase = 0, issued = 0;
             bool alive = true;
+            const uint64_t policy = evict_first_policy();
             // Units are claimed from a device-wide counter, so a CTA that starts early or meets
             // short units simply takes more of them.  The claim for the NEXT unit and its row
             // count are requested before the current unit is streamed, so neither round trip
@@ -459,7 +472,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                         if (!wait(&sh->empty[stage], phase ^ 1)) { alive = false; break; }
                         const uint32_t bytes = (uint32_t)min(CR, cnt - r0) * ROWB;
                         tc::mbar_arrive_expect_tx(&sh->full[stage], bytes);
-                        bulk_load(ring + stage * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[stage]);
+                        bulk_load(ring + stage * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[stage], policy);
                         ++issued;
                         if (++stage == kStreamStages) { stage = 0; phase ^= 1; }
                     }
