@@ -60,7 +60,14 @@ typedef struct a2sf_params {
     int32_t budget, recent;
     float alpha;
     float scale;
+    int32_t flags;               /* 0 or A2SF_FLAG_* */
 } a2sf_params;
+
+/* Scoring pass: Eq. 5 weighs query row i with alpha^(n-1-i).  Once that weight is below
+ * 2^-127 (2^-152 on the CUDA-core path) the fp32 term is exactly zero, so with this flag the
+ * pass leaves those rows out: O(n * window) instead of O(n^2) work with bit-identical scores.
+ * Off by default; alpha = 1 has no such rows. */
+#define A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS 1
 
 typedef struct a2sf_cache a2sf_cache;   /* opaque, owned by the library */
 

@@ -25,7 +25,7 @@ A2SF_ERR_TIMEOUT, A2SF_ERR_WORKSPACE = -4, -5
 class a2sf_params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("budget", ctypes.c_int32), ("recent", ctypes.c_int32),
-                ("alpha", ctypes.c_float), ("scale", ctypes.c_float)]
+                ("alpha", ctypes.c_float), ("scale", ctypes.c_float), ("flags", ctypes.c_int32)]
 
 
 class A2SFError(RuntimeError):
@@ -101,9 +101,12 @@ def _stream(stream) -> ctypes.c_void_p:
     return ctypes.c_void_p(stream.cuda_stream)
 
 
+A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS = 1
+
+
 def make_params(B: int, H: int, d: int, dtype: torch.dtype, budget: int, recent: int,
-                alpha: float, scale: float = 0.0) -> a2sf_params:
-    return a2sf_params(B, H, d, _DTYPE_CODE[dtype], budget, recent, alpha, scale)
+                alpha: float, scale: float = 0.0, flags: int = 0) -> a2sf_params:
+    return a2sf_params(B, H, d, _DTYPE_CODE[dtype], budget, recent, alpha, scale, flags)
 
 
 def a2sf_kernel_launch_count() -> int:

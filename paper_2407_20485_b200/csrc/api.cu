@@ -27,6 +27,7 @@ static int check_params(const a2sf_params *p)
         return A2SF_ERR_UNSUPPORTED;
     if (p->d != 64 && p->d != 128) return A2SF_ERR_UNSUPPORTED;
     if ((int64_t)p->B * p->H > 0x7fffffff) return A2SF_ERR_INVALID_ARG;
+    if (p->flags & ~A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) return A2SF_ERR_INVALID_ARG;
     return A2SF_OK;
 }
 
@@ -113,6 +114,7 @@ static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
+    a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
     a.v_half = nullptr; a.v_flag = nullptr;
     if (prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d) > 0) {
         char *extra = static_cast<char *>(workspace) + align_up((size_t)p->B * p->H * n * sizeof(float));
@@ -162,6 +164,7 @@ static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.st = Strides{stride_b, stride_h, stride_t};
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
+    a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
     a.v_half = nullptr; a.v_flag = nullptr;
     return run_scores_and_select(p, n, a, kept_idx, static_cast<cudaStream_t>(cuda_stream));
 }

@@ -170,8 +170,15 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
     const float neg_log2_alpha = alpha > 0.f ? -log2f(alpha) : INFINITY;
     const float sl2 = a.scale * kLog2e;
 
+    // rows whose weight is below 2^-152 contribute exactly 0 even with denormals
+    int i_first = kb * kRows;
+    if (a.skip_zero_rows && neg_log2_alpha > 0.f) {
+        const float span = ceilf(152.f / neg_log2_alpha);
+        const int i_min = span >= (float)a.n ? 0 : min(a.n - 1, a.n - (int)span);
+        i_first = max(i_first, (i_min / kTile) * kTile);
+    }
     float acc = 0.f;
-    for (int i0 = kb * kRows; i0 < a.n; i0 += kTile) {
+    for (int i0 = i_first; i0 < a.n; i0 += kTile) {
         __syncthreads();
         load_tile<T, D>(Qs, Q, a.st.t, i0, a.n);
         if (threadIdx.x < kTile) {

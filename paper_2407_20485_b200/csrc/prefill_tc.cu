@@ -41,6 +41,7 @@ struct ScoreArgs {
     float sl2;            // scale * log2(e)
     float alpha;          // forgetting factor, or per unit:
     const float *alpha_vec;
+    int skip_zero_rows;   // leave out query tiles whose forgetting weight underflows to exactly 0
 };
 
 struct ScoreShared {
@@ -102,7 +103,17 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
     const int ntile_total = (a.n + kBlk - 1) / kBlk;
     const int u = blockIdx.x / ntile_total, kb = blockIdx.x % ntile_total;
     const int b = u / a.H, h = u % a.H;
-    const int ntiles = ntile_total - kb;               // query-row tiles kb .. last
+    // Rows older than 127/(-log2 alpha) carry a weight below 2^-127: their flushed fp32
+    // exponential is exactly 0, so leaving their tiles out changes no bit of the result.
+    const float alpha = unit_alpha(a.alpha_vec, u, a.alpha);
+    const float neg_log2_alpha = alpha > 0.f ? -log2f(alpha) : INFINITY;   // alpha = 0: only row n-1
+    int t_first = kb;
+    if (a.skip_zero_rows && neg_log2_alpha > 0.f) {
+        const float span = ceilf(127.f / neg_log2_alpha);                  // first age with weight 0
+        const int i_min = span >= (float)a.n ? 0 : min(a.n - 1, a.n - (int)span);
+        t_first = max(kb, i_min / kBlk);
+    }
+    const int ntiles = ntile_total - t_first;          // query-row tiles t_first .. last
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sh->abort_flag;
 
@@ -141,8 +152,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
                 if (!mbar_wait(&sh->q_empty[s], ph ^ 1, abort_flag)) break;
                 mbar_arrive_expect_tx(&sh->q_full[s], kTileBytes);
                 uint8_t *dst = Qs + s * kTileBytes;
-                tma_load_4d(dst, &tmap_q, &sh->q_full[s], 0, (kb + it) * kBlk, h, b);
-                tma_load_4d(dst + kHalfBytes, &tmap_q, &sh->q_full[s], 64, (kb + it) * kBlk, h, b);
+                tma_load_4d(dst, &tmap_q, &sh->q_full[s], 0, (t_first + it) * kBlk, h, b);
+                tma_load_4d(dst + kHalfBytes, &tmap_q, &sh->q_full[s], 64, (t_first + it) * kBlk, h, b);
                 issued = it + 1;
             }
             if (*abort_flag) {
@@ -182,8 +193,6 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         const int j = kb * kBlk + key_lane;
         const int et = threadIdx.x - 64;            // 0..255
         const float *lse = a.lse + (size_t)u * a.n;
-        const float alpha = unit_alpha(a.alpha_vec, u, a.alpha);
-        const float neg_log2_alpha = alpha > 0.f ? -log2f(alpha) : INFINITY;   // alpha = 0: only row n-1
         // A failed wait poisons the CTA: later waits return at once and the loop keeps its
         // shape, so every thread still reaches the final barrier; the status word reports it.
         auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
@@ -198,12 +207,12 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             const int age = a.n - 1 - i;
             return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha);
         };
-        float c_next = hsel == 0 ? row_const(kb * kBlk + et) : 0.f;
+        float c_next = hsel == 0 ? row_const(t_first * kBlk + et) : 0.f;
         float sum = 0.f;
         for (int it = 0; it < ntiles; ++it) {
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
-            const int i0 = (kb + it) * kBlk;
+            const int i0 = (t_first + it) * kBlk;
             if (hsel == 0) sh->cbuf[it & 1][et] = c_next;
             // every epilogue thread arrives: the constants are published, and nobody is still
             // reading the buffer that the tile after next will overwrite
@@ -213,7 +222,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             wait(&sh->acc_full[acc], aph);
             tc_fence_after_sync();
             const float *cb = sh->cbuf[it & 1] + hsel * 64;
-            const bool diag = (it == 0);
+            const bool diag = (t_first + it == kb);
             // this thread's 64-row strip comes into registers with one wait, and the
             // accumulator buffer goes back to the tensor core before the arithmetic starts
             uint32_t r[2][32];
@@ -794,6 +803,7 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     sa.sl2 = a.scale * kLog2e;
     sa.alpha = a.alpha;
     sa.alpha_vec = a.alpha_vec;
+    sa.skip_zero_rows = a.skip_zero_rows;
     const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
     score_pass_tc<<<grid, kScoreThreads, kScoreSmemBytes, s>>>(mq, mk, sa, dtype == A2SF_BF16 ? 1 : 0);
     count_launch();

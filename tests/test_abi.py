@@ -56,7 +56,7 @@ def test_size_queries_need_no_gpu(a2sf):
 @pytest.mark.parametrize("field,value,status", [
     ("d", 96, -2), ("dtype", 7, -2), ("budget", 0, -1), ("recent", 600, -1), ("recent", -1, -1),
     ("alpha", 1.5, -1), ("alpha", -0.1, -1), ("alpha", float("nan"), -1), ("B", 0, -1),
-    ("scale", -1.0, -1),
+    ("scale", -1.0, -1), ("flags", 8, -1),
 ])
 def test_bad_parameters_are_rejected_on_the_host(a2sf, field, value, status):
     import torch

@@ -195,6 +195,38 @@ def test_export_import_round_trip_and_generator_on_device():
     assert a2sf.a2sf_kernel_launch_count() > 0
 
 
+# ---- scoring pass that leaves out rows whose forgetting weight is exactly zero ------------------
+@pytest.mark.parametrize("name,kw,alphas", [
+    ("llama2_13b", dict(B=1, H=3, n=1100), [0.5, 0.9, 0.0, 1.0, 0.3]),      # tensor-core pass
+    ("opt_6p7b", dict(B=1, H=2, n=777), [0.1, 0.97]),
+    ("tiny_fp32", dict(H=3, n=700, budget=64, recent=16), [0.5, 0.0, 1.0, 0.8]),   # CUDA-core pass
+])
+def test_zero_weight_rows_can_be_skipped_without_changing_a_bit(name, kw, alphas):
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(steps=0, **kw)
+    q, k, v = (t.cuda() for t in wl.make_prompt(w))
+    for al in alphas:
+        p0 = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, al)
+        p1 = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, al,
+                              flags=a2sf.A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS)
+        out0, S0, kept0, lse0 = a2sf.a2sf_prefill(p0, q, k, v)
+        out1, S1, kept1, lse1 = a2sf.a2sf_prefill(p1, q, k, v)
+        S2, kept2 = a2sf.a2sf_rescore(p1, q, k, lse0)
+        torch.cuda.synchronize()
+        assert torch.equal(S0, S1) and torch.equal(kept0, kept1) and torch.equal(out0, out1), al
+        assert torch.equal(S0, S2) and torch.equal(kept0, kept2), al
+    # per-head factors: every unit uses its own window
+    av = torch.tensor([0.0, 0.2, 0.9, 1.0, 0.5, 0.7], dtype=torch.float32)[torch.arange(w.units) % 6].cuda()
+    p0 = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, 0.5)
+    p1 = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, 0.5,
+                          flags=a2sf.A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS)
+    _, S0, kept0, _ = a2sf.a2sf_prefill(p0, q, k, v, alphas=av.view(w.B, w.H))
+    _, S1, kept1, _ = a2sf.a2sf_prefill(p1, q, k, v, alphas=av.view(w.B, w.H))
+    torch.cuda.synchronize()
+    assert torch.equal(S0, S1) and torch.equal(kept0, kept1)
+
+
 # ---- one forgetting factor per head (the paper's Limitation section) -------------------------
 @pytest.mark.parametrize("name,kw", [
     ("llama2_7b", dict(B=2, H=3, n=500, steps=30)),              # tensor-core prefill, streaming decode
