@@ -33,6 +33,10 @@ constexpr int kTileBytes = 2 * kHalfBytes;  // 32 KB
 constexpr int kScoreStages = 2;
 constexpr int kScoreThreads = 320;           // producer warp, MMA warp, 8 epilogue warps
 constexpr int kScoreEpiThreads = 256;
+// Ring of row-constant vectors written by the producer warp.  Slot x%ring is rewritten for tile x
+// after the MMAs of tile x-2 have retired; those needed the accumulator that tile x-4 held, i.e.
+// every epilogue thread had finished the arithmetic of tile x-5.  Any depth >= 5 is safe.
+constexpr int kScoreCRing = 8;
 
 struct ScoreArgs {
     const float *lse;     // [U][n]
@@ -45,10 +49,11 @@ struct ScoreArgs {
 };
 
 struct ScoreShared {
-    uint64_t k_full, q_full[kScoreStages], q_empty[kScoreStages], acc_full[2], acc_empty[2], c_full[2];
+    uint64_t k_full, q_full[kScoreStages], q_empty[kScoreStages], acc_full[2], acc_empty[2];
+    uint64_t c_ready[kScoreCRing];
     uint32_t tmem_base;
     int abort_flag;
-    float cbuf[2][kBlk];
+    float cbuf[kScoreCRing][kBlk];   // row constants of the query tiles in flight
     float part[kBlk];           // upper-half partial sums, added to the lower half at the end
 };
 
@@ -79,6 +84,30 @@ __device__ __forceinline__ void issue_qk_mma(uint32_t d_tmem, uint64_t a_desc, u
         const uint64_t off = (uint64_t)(((k >> 2) * kHalfBytes + (k & 3) * 32) >> 4);
         umma_ss(d_tmem, a_desc + off, b_desc + off, idesc, k > 0);
     }
+}
+
+// Sum of exp2(s*sl2 - c_i) over this thread's 64 query rows of the tile.  Masked: rows
+// below `first_row` (relative to the strip) lie above the diagonal and contribute nothing.
+template <bool Masked>
+__device__ __forceinline__ float strip_sum(const uint32_t (&r)[2][32], const float *cb, float sl2,
+                                           int first_row)
+{
+    float part[4] = {0.f, 0.f, 0.f, 0.f};           // four independent add chains
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+#pragma unroll
+        for (int x = 0; x < 32; x += 4) {
+            const float4 c4 = *reinterpret_cast<const float4 *>(cb + c * 32 + x);
+            const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float pw = ex2_approx(fmaf(__uint_as_float(r[c][x + e]), sl2, -cc[e]));
+                if (Masked) pw = (c * 32 + x + e >= first_row) ? pw : 0.f;   // rows i >= j
+                part[e] += pw;
+            }
+        }
+    }
+    return (part[0] + part[1]) + (part[2] + part[3]);
 }
 
 __global__ void __launch_bounds__(kScoreThreads, 2)
@@ -123,8 +152,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sh->acc_full[x], 1);
             mbar_init(&sh->acc_empty[x], kScoreEpiThreads);
-            mbar_init(&sh->c_full[x], kScoreEpiThreads);
         }
+        for (int x = 0; x < kScoreCRing; ++x) mbar_init(&sh->c_ready[x], 1);
         sh->abort_flag = 0;
         fence_mbar_init();
     }
@@ -138,31 +167,56 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
     const uint32_t tmem_base = sh->tmem_base;
 
     if (warp == 0) {
-        // ---- TMA producer ---------------------------------------------------------
+        // ---- TMA producer; its 32 lanes also prepare the row constants ------------------
+        //   c_i = lse_i*log2e + (n-1-i)*(-log2 alpha);  rows past n give +inf (weight 0).
+        // They are written one tile ahead of the tensor core, so the epilogue warps never meet
+        // at a barrier of their own and drift freely against each other.
+        const float *lse = a.lse + (size_t)u * a.n;
         if (lane == 0) {
             prefetch_tmap(&tmap_q);
             prefetch_tmap(&tmap_k);
             mbar_arrive_expect_tx(&sh->k_full, kTileBytes);
             tma_load_4d(Ks, &tmap_k, &sh->k_full, 0, kb * kBlk, h, b);
             tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full, 64, kb * kBlk, h, b);
-            int issued = 0;
-            for (int it = 0; it < ntiles; ++it) {
-                const int s = it % kScoreStages;
-                const uint32_t ph = (it / kScoreStages) & 1;
-                if (!mbar_wait(&sh->q_empty[s], ph ^ 1, abort_flag)) break;
-                mbar_arrive_expect_tx(&sh->q_full[s], kTileBytes);
-                uint8_t *dst = Qs + s * kTileBytes;
-                tma_load_4d(dst, &tmap_q, &sh->q_full[s], 0, (t_first + it) * kBlk, h, b);
-                tma_load_4d(dst + kHalfBytes, &tmap_q, &sh->q_full[s], 64, (t_first + it) * kBlk, h, b);
-                issued = it + 1;
+        }
+        int issued = 0;
+        for (int it = 0; it < ntiles; ++it) {
+            const int s = it % kScoreStages;
+            const uint32_t ph = (it / kScoreStages) & 1;
+            const int i0 = (t_first + it) * kBlk;
+            // the constants' global loads are in flight while lane 0 waits for the stage
+            float c4[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int i = i0 + lane * 4 + e;
+                const int age = a.n - 1 - i;
+                c4[e] = i < a.n ? fmaf(__ldg(lse + i), kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha)
+                                : INFINITY;
             }
-            if (*abort_flag) {
-                // give copies still in flight a bounded chance to land before the CTA exits
-                int dummy = 0;
-                for (int it = max(0, issued - kScoreStages); it < issued; ++it)
-                    mbar_wait(&sh->q_full[it % kScoreStages], (it / kScoreStages) & 1, &dummy);
-                mbar_wait(&sh->k_full, 0, &dummy);
+            int ok = 1;
+            if (lane == 0) {
+                ok = mbar_wait(&sh->q_empty[s], ph ^ 1, abort_flag) ? 1 : 0;
+                if (ok) {
+                    mbar_arrive_expect_tx(&sh->q_full[s], kTileBytes);
+                    uint8_t *dst = Qs + s * kTileBytes;
+                    tma_load_4d(dst, &tmap_q, &sh->q_full[s], 0, i0, h, b);
+                    tma_load_4d(dst + kHalfBytes, &tmap_q, &sh->q_full[s], 64, i0, h, b);
+                }
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            issued = it + 1;
+            *reinterpret_cast<float4 *>(&sh->cbuf[it % kScoreCRing][lane * 4]) =
+                make_float4(c4[0], c4[1], c4[2], c4[3]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->c_ready[it % kScoreCRing]);
+        }
+        if (lane == 0 && *abort_flag) {
+            // give copies still in flight a bounded chance to land before the CTA exits
+            int dummy = 0;
+            for (int it = max(0, issued - kScoreStages); it < issued; ++it)
+                mbar_wait(&sh->q_full[it % kScoreStages], (it / kScoreStages) & 1, &dummy);
+            mbar_wait(&sh->k_full, 0, &dummy);
         }
     } else if (warp == 1) {
         // ---- MMA issuer -------------------------------------------------------------
@@ -191,37 +245,21 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         const int hsel = (warp - 2) >> 2;           // which half of the tile's query rows
         const int key_lane = quarter * 32 + lane;
         const int j = kb * kBlk + key_lane;
-        const int et = threadIdx.x - 64;            // 0..255
-        const float *lse = a.lse + (size_t)u * a.n;
         // A failed wait poisons the CTA: later waits return at once and the loop keeps its
         // shape, so every thread still reaches the final barrier; the status word reports it.
         auto wait = [&](uint64_t *bar, uint32_t parity) -> bool {
             if (*abort_flag) return false;
             return mbar_wait(bar, parity, abort_flag);
         };
-        // row constant c_i = lse_i*log2e + (n-1-i)*(-log2 alpha); rows past n give +inf.
-        // The value for the NEXT tile is requested one tile ahead so its global-memory latency
-        // never sits between two tiles.  The lower-half threads publish the 128 constants.
-        auto row_const = [&](int i) -> float {
-            if (i >= a.n) return INFINITY;
-            const int age = a.n - 1 - i;
-            return fmaf(lse[i], kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha);
-        };
-        float c_next = hsel == 0 ? row_const(t_first * kBlk + et) : 0.f;
         float sum = 0.f;
         for (int it = 0; it < ntiles; ++it) {
             const int acc = it & 1;
             const uint32_t aph = (it >> 1) & 1;
             const int i0 = (t_first + it) * kBlk;
-            if (hsel == 0) sh->cbuf[it & 1][et] = c_next;
-            // every epilogue thread arrives: the constants are published, and nobody is still
-            // reading the buffer that the tile after next will overwrite
-            mbar_arrive(&sh->c_full[acc]);
-            if (hsel == 0 && it + 1 < ntiles) c_next = row_const(i0 + kBlk + et);
-            wait(&sh->c_full[acc], aph);
+            wait(&sh->c_ready[it % kScoreCRing], (it / kScoreCRing) & 1);
             wait(&sh->acc_full[acc], aph);
             tc_fence_after_sync();
-            const float *cb = sh->cbuf[it & 1] + hsel * 64;
+            const float *cb = sh->cbuf[it % kScoreCRing] + hsel * 64;
             const bool diag = (t_first + it == kb);
             // this thread's 64-row strip comes into registers with one wait, and the
             // accumulator buffer goes back to the tensor core before the arithmetic starts
@@ -232,22 +270,10 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             tmem_wait_ld();
             tc_fence_before_sync();
             mbar_arrive(&sh->acc_empty[acc]);
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                float part = 0.f;
-#pragma unroll
-                for (int x = 0; x < 32; x += 4) {
-                    const float4 c4 = *reinterpret_cast<const float4 *>(cb + c * 32 + x);
-                    const float cc[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        float pw = ex2_approx(fmaf(__uint_as_float(r[c][x + e]), a.sl2, -cc[e]));
-                        if (diag) pw = (i0 + hsel * 64 + c * 32 + x + e >= j) ? pw : 0.f;   // rows i >= j
-                        part += pw;
-                    }
-                }
-                sum += part;
-            }
+            // only the diagonal tile needs the causal test; the others run the bare
+            // multiply-add / exponential / add per logit
+            if (diag) sum += strip_sum<true>(r, cb, a.sl2, j - (i0 + hsel * 64));
+            else      sum += strip_sum<false>(r, cb, a.sl2, 0);
         }
         if (hsel == 1) sh->part[key_lane] = sum;
         named_barrier(1, kScoreEpiThreads);
