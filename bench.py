@@ -297,9 +297,73 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(w, T, q, k, v, dq, dk, dv)
     cache.close()
+    if rank == 0 and world == 1 and not args.no_rotation:
+        # the other stated workloads: their one-layer caches fit in L2, so they are also
+        # stepped as a rotation over the named model's layer count (not part of the headline)
+        result["decode_layer_rotation"] = [
+            decode_layer_rotation(a2sf, dev, name, layers, args.rotation_steps, args.rotation_reps)
+            for name, layers in (("llama2_7b", 32), ("opt_6p7b", 32), ("long_context", 32))]
     if rank == 0:
         print(json.dumps(result))
     a2dist.finalize()
+
+
+def decode_layer_rotation(a2sf, dev, name, layers, steps, reps):
+    """Decode-step timing for a workload whose single-layer cache fits in L2: `layers`
+    independent cache instances (the layer count of the named model) are stepped round-robin, so
+    the working set is what one generation step of the whole model touches.  `steps` x `layers`
+    launches are captured once in a CUDA graph; each repetition restores every cache (untimed)
+    and times one replay with CUDA events.  Also run with one layer (L2-resident) for contrast."""
+    w = wl.WORKLOADS[name]
+    q, k, v = wl.make_prompt_chunked(w, dev)
+    dq, dk, dv = wl.make_decode(w, dev, t_range=(0, steps))
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    _, S, kept, _ = a2sf.a2sf_prefill(p, q, k, v)
+    del q
+    bytes_per_launch = w.units * w.decode_bytes_per_unit_step()
+    res = {"workload": f"{w.name} (config {w.index}): B{w.B} H{w.H} d{w.d} n{w.n} alpha{w.alpha} "
+                       f"budget{w.budget} recent{w.recent}",
+           "bytes_per_launch": bytes_per_launch, "steps_per_replay": steps, "repetitions": reps,
+           "timing": "one CUDA-graph replay of steps x layers launches between two events"}
+    for L in (1, layers):
+        caches = [a2sf.Cache(p, dev) for _ in range(L)]
+        o = torch.empty((L, w.B, w.H, w.d), dtype=w.torch_dtype, device=dev)
+        e = torch.empty((L, w.B, w.H), dtype=torch.int32, device=dev)
+
+        def restore():
+            for c in caches:
+                c.a2sf_cache_load(k, v, S, kept)
+
+        def run():
+            for t in range(steps):
+                for l, c in enumerate(caches):
+                    c.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o[l], e[l])
+
+        restore(); run()                        # lazy initialisation happens outside the capture
+        torch.cuda.synchronize()
+        restore()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            run()
+        times = []
+        for _ in range(reps):
+            restore()
+            ev = cuda_events(2)
+            ev[0].record(); g.replay(); ev[1].record()
+            torch.cuda.synchronize()
+            times.append(ev[0].elapsed_time(ev[1]) * 1e3 / (steps * L))      # us per launch
+        assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+        med, best = statistics.median(times), min(times)
+        res["layers_%d" % L] = {
+            "working_set_mb": L * bytes_per_launch / 1e6,
+            "l2": "larger_than_l2" if L * bytes_per_launch > 126e6 else "l2_resident",
+            "us_per_launch_median": med, "us_per_launch_min": best,
+            "gbps_median": bytes_per_launch / med / 1e3, "gbps_max": bytes_per_launch / best / 1e3}
+        del g
+        for c in caches:
+            c.close()
+    return res
 
 
 def oracle_sample(w, units_sel, dsteps, q, k, v, dq, dk, dv, threads):
@@ -416,6 +480,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-rotation", action="store_true",
+                    help="skip the layer-rotation decode timing of the L2-resident workloads")
+    ap.add_argument("--rotation-steps", type=int, default=16, help="decode steps per graph replay")
+    ap.add_argument("--rotation-reps", type=int, default=10)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -195,6 +195,52 @@ def test_export_import_round_trip_and_generator_on_device():
     assert a2sf.a2sf_kernel_launch_count() > 0
 
 
+# ---- the calls are asynchronous and hold no host-side state: a captured graph replays them ------
+@pytest.mark.parametrize("name,kw", [
+    ("llama2_7b", dict(H=6, n=400, steps=12)),                                  # streaming kernel
+    ("long_context", dict(H=2, n=1500, budget=1024, recent=512, steps=12)),    # cluster split-K
+])
+def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches(name, kw):
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    dq, dk, dv = wl.make_decode(w, device="cuda")
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    _, S, kept, _ = a2sf.a2sf_prefill(p, q, k, v)
+    direct, graphed = a2sf.Cache(p), a2sf.Cache(p)
+    T = w.steps
+    o1 = torch.empty((T, w.B, w.H, w.d), dtype=q.dtype, device="cuda")
+    o2 = torch.empty_like(o1)
+    e1 = torch.empty((T, w.B, w.H), dtype=torch.int32, device="cuda")
+    e2 = torch.empty_like(e1)
+    direct.a2sf_cache_load(k, v, S, kept)
+    for t in range(T):
+        direct.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o1[t], e1[t])
+    graphed.a2sf_cache_load(k, v, S, kept)
+    graphed.a2sf_decode_step(w.alpha, dq[0], dk[0], dv[0], o2[0], e2[0])   # lazy set-up, uncaptured
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for t in range(T):
+            graphed.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o2[t], e2[t])
+    for _ in range(2):                     # the same graph, twice, from the same restored state
+        graphed.a2sf_cache_load(k, v, S, kept)
+        o2.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(o1, o2) and torch.equal(e1, e2)
+        s1, s2 = direct.a2sf_cache_export(), graphed.a2sf_cache_export()
+        torch.cuda.synchronize()
+        c = s1["count"].flatten()
+        assert torch.equal(s1["count"], s2["count"]) and torch.equal(s1["len"], s2["len"])
+        for key in ("scores", "pos"):
+            a_, b_ = s1[key].flatten(0, 1), s2[key].flatten(0, 1)
+            for u in range(w.units):
+                assert torch.equal(a_[u, :c[u]], b_[u, :c[u]])
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+
+
 # ---- scoring pass that leaves out rows whose forgetting weight is exactly zero ------------------
 @pytest.mark.parametrize("name,kw,alphas", [
     ("llama2_13b", dict(B=1, H=3, n=1100), [0.5, 0.9, 0.0, 1.0, 0.3]),      # tensor-core pass
