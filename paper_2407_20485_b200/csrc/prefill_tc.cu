@@ -67,6 +67,13 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
+
 // The issuing thread is the bottleneck of small-tile UMMA pipelines, so descriptors are built
 // once per operand buffer and only advanced by a constant per K-step.
 __device__ __forceinline__ uint64_t kmajor_desc(uint32_t smem_addr)
@@ -331,10 +338,13 @@ struct AttnShared {
     uint64_t s_full[2], p_full[2], o_done[2];       // per stream
     uint32_t tmem_base;
     int abort_flag;
+    float xch[2][2][kBlk];                          // [stream][column half][row]: row maxima / sums
 };
 
-// Q_A, Q_B, K ring, V ring
-constexpr size_t kAttnSmemBytes = 1024 + kTileBytes * (2 + kKStages + kVStages) + sizeof(AttnShared);
+// Q_A, Q_B, K ring, V ring.  The kernel has no static shared memory and declares the dynamic
+// array 1024-byte aligned (the 128-byte swizzle pattern repeats every 1024 bytes), so no slack
+// is added: the seven tiles leave 3 KB for the barriers and the exchange buffer.
+constexpr size_t kAttnSmemBytes = kTileBytes * (2 + kKStages + kVStages) + sizeof(AttnShared);
 static_assert(kAttnSmemBytes <= 227 * 1024, "attention pass shared memory");
 
 template <typename T> __device__ __forceinline__ uint32_t pack2(float a, float b);
@@ -359,18 +369,20 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
              const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
 {
     // once any CTA has given up on a wait, the rest of the grid drains without working
-    __shared__ int s_skip;
-    if (threadIdx.x == 0) {
-        int skip = *reinterpret_cast<volatile int *>(&g_tc_status);
-        if (a.v_flag && (*a.v_flag != 0) != (a.run_if_flag != 0)) skip = 1;   // the other launch's job
-        s_skip = skip;
+    extern __shared__ __align__(1024) uint8_t attn_smem[];
+    {
+        int skip = 0;
+        if (threadIdx.x == 0) {
+            skip = *reinterpret_cast<volatile int *>(&g_tc_status);
+            if (a.v_flag && (*a.v_flag != 0) != (a.run_if_flag != 0)) skip = 1;   // the other launch's job
+            if (smem_u32(attn_smem) & 1023u) {           // the swizzled tiles need this alignment
+                g_tc_status = A2SF_ERR_CUDA;
+                skip = 1;
+            }
+        }
+        if (__syncthreads_or(skip)) return;
     }
-    __syncthreads();
-    if (s_skip) return;
-
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                                ~uintptr_t(1023));
+    uint8_t *smem = attn_smem;
     uint8_t *Qs = smem;                                  // two tiles: stream A, stream B
     uint8_t *Ks = smem + 2 * kTileBytes;
     uint8_t *Vs = Ks + kKStages * kTileBytes;
@@ -406,7 +418,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         for (int s = 0; s < kVStages; ++s) { mbar_init(&sh->v_full[s], 1); mbar_init(&sh->v_empty[s], 1); }
         for (int x = 0; x < 2; ++x) {
             mbar_init(&sh->s_full[x], 1);
-            mbar_init(&sh->p_full[x], kBlk);
+            mbar_init(&sh->p_full[x], 2 * kBlk);
             mbar_init(&sh->o_done[x], 1);
         }
         sh->abort_flag = 0;
@@ -483,14 +495,19 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             auto issue_pv = [&](int X, int t) {
                 const uint64_t vd = v_desc[t % kVStages];
                 const uint32_t sp = tmem_base + X * 2 * kBlk, o = sp + kBlk;
-                // 16 keys per step: 8 columns of packed P; two 8-key groups of V = 2048 bytes
+                // 16 keys per step: 8 columns of packed P; two 8-key groups of V = 2048 bytes.
+                // Keys 64h .. 64h+63 have their P at columns 64h .. 64h+31 (second term of the
+                // two-term form at 64h+32 .. 64h+63): each softmax thread writes only over the
+                // logits columns it has read itself.
 #pragma unroll
                 for (int k = 0; k < kBlk / 16; ++k)
-                    umma_ts(o, sp + k * 8, vd + (uint64_t)(k * 2048 >> 4), idesc_pv, (t > 0) || (k > 0));
+                    umma_ts(o, sp + 64 * (k >> 2) + 8 * (k & 3), vd + (uint64_t)(k * 2048 >> 4), idesc_pv,
+                            (t > 0) || (k > 0));
                 if (kSplitP) {
 #pragma unroll
                     for (int k = 0; k < kBlk / 16; ++k)
-                        umma_ts(o, sp + kBlk / 2 + k * 8, vd + (uint64_t)(k * 2048 >> 4), idesc_pv, 1);
+                        umma_ts(o, sp + 64 * (k >> 2) + 32 + 8 * (k & 3), vd + (uint64_t)(k * 2048 >> 4),
+                                idesc_pv, 1);
                 }
                 umma_commit(&sh->o_done[X]);
             };
@@ -521,48 +538,56 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
             }
         }
     } else {
-        // ---- softmax + epilogue: one thread per query row of its stream --------------------
-        const int X = (warp - 2) >> 2;                     // stream
-        const int ntX = X == 0 ? ntA : ntB;
+        // ---- softmax + epilogue: two threads per query row, the streams taken in turn --------
+        // All eight warps work on one stream's tile at a time, each thread on 64 of its row's
+        // 128 logits, so a tile spends half as long between its two MMAs as with one thread per
+        // row; the other stream's MMAs fill that time.
         const int quarter = warp & 3;                      // TMEM lanes this warp may touch
+        const int half = (warp - 2) >> 2;                  // columns 64*half .. 64*half+63
         const int r = quarter * 32 + lane;                 // row in the tile = TMEM lane
-        const int i = (X == 0 ? rbA : rbB) * kBlk + r;
-        const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-        const uint32_t sp = tmem_base + X * 2 * kBlk + lane_off;   // logits, then P hi | P lo
-        const uint32_t to = sp + kBlk;                             // output accumulator
-        float m_used = 0.f, l = 0.f;
-        for (int t = 0; t < ntX; ++t) {
+        const uint32_t lane_off = ((uint32_t)(quarter * 32) << 16) + half * 64;
+        float m_used[2] = {0.f, 0.f}, l[2] = {0.f, 0.f};   // per stream; l covers this thread's columns
+        auto do_tile = [&](auto Xc, int t, int ntX) {
+            constexpr int X = decltype(Xc)::value;
+            const uint32_t sp = tmem_base + X * 2 * kBlk + lane_off;   // own logits, then own P
+            const uint32_t to = sp + kBlk;                             // own half of the accumulator
             wait(&sh->s_full[X], t & 1);
             tc_fence_after_sync();
-            const bool diag = (t == ntX - 1);
-            // pass 1: row maximum of the raw logits.  Only the diagonal tile pays for the mask.
-            float smax = -INFINITY;
-            auto row_max = [&](auto masked) {
-                // all four loads are in flight before the single wait
-                uint32_t v[4][32];
+            // the thread's 64 logits come into registers once and serve both passes
+            uint32_t v[2][32];
+            tmem_ld32(sp, v[0]);
+            tmem_ld32(sp + 32, v[1]);
+            tmem_wait_ld();
+            if (t == ntX - 1) {
+                // diagonal tile: a masked logit becomes -inf, whose exponential is exactly 0
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(sp + c * 32, v[c]);
-                tmem_wait_ld();
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                    for (int x = 0; x < 32; ++x)
+                        if (half * 64 + c * 32 + x > r) v[c][x] = 0xff800000u;
+            }
+            // pass 1: row maximum; the two threads of a row exchange theirs through shared memory
+            float mx[2];
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) {
-                        float sv = __uint_as_float(v[c][x]);
-                        if (decltype(masked)::value && c * 32 + x > r) sv = -INFINITY;   // causal mask
-                        mx[c] = fmaxf(mx[c], sv);
-                    }
-                smax = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            };
-            if (diag) row_max(std::true_type{}); else row_max(std::false_type{});
+            for (int c = 0; c < 2; ++c) {
+                mx[c] = max3(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]), __uint_as_float(v[c][2]));
+#pragma unroll
+                for (int x = 3; x + 1 < 32; x += 2)
+                    mx[c] = max3(mx[c], __uint_as_float(v[c][x]), __uint_as_float(v[c][x + 1]));
+                mx[c] = fmaxf(mx[c], __uint_as_float(v[c][31]));
+            }
+            const float own = fmaxf(mx[0], mx[1]);
+            sh->xch[X][half][r] = own;
+            named_barrier(1 + quarter, 64);                // this quarter's two warps
+            const float smax = fmaxf(own, sh->xch[X][half ^ 1][r]);
             // Lazy maximum (log2 domain): the reference moves only on the first tile or when
             // the row maximum exceeds it by more than 2^8; otherwise probabilities up to 256
-            // are simply kept.
-            const float xmax = fmaf(smax, a.sl2, -m_used);
+            // are simply kept.  Both threads of a row see the same smax and decide alike.
+            const float xmax = fmaf(smax, a.sl2, -m_used[X]);
             const bool grow = (t == 0) || (xmax > kRescaleThreshold);
             float factor = 1.f;
             if (grow) {
-                m_used += xmax;
+                m_used[X] += xmax;
                 factor = t == 0 ? 0.f : ex2_approx(-xmax);
             }
             if (t > 0 && __any_sync(0xffffffffu, grow)) {
@@ -570,7 +595,7 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 wait(&sh->o_done[X], (t - 1) & 1);
                 tc_fence_after_sync();
 #pragma unroll 1
-                for (int c = 0; c < kD / 32; ++c) {
+                for (int c = 0; c < 2; ++c) {
                     uint32_t o[32];
                     tmem_ld32(to + c * 32, o);
                     tmem_wait_ld();
@@ -580,84 +605,72 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 }
                 tmem_wait_st();
             }
-            // pass 2: probabilities; P overwrites the logits columns.  32 logits columns become
-            // 16 columns of P (high part at [16c, 16c+16), low part at [64+16c, 80+16c)).  The
-            // high part only lands on columns already read; the low parts of the first three
-            // chunks are held back until their destination columns have been read.
-            const float neg_m = -m_used;
-            float rowsum = 0.f;
-            auto write_p = [&](auto masked) {
-                uint32_t lo_hold[3][16];
+            // pass 2: probabilities, packed in pairs over the thread's own logits columns
+            const float neg_m = -m_used[X];
+            float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(sp + c * 32, v);
-                    tmem_wait_ld();
-                    uint32_t hi[16], lo[16];
+            for (int c = 0; c < 2; ++c) {
+                uint32_t hi[16], lo[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        float p0 = ex2_approx(fmaf(__uint_as_float(v[2 * e]), a.sl2, neg_m));
-                        float p1 = ex2_approx(fmaf(__uint_as_float(v[2 * e + 1]), a.sl2, neg_m));
-                        if (decltype(masked)::value) {
-                            if (c * 32 + 2 * e > r) p0 = 0.f;
-                            if (c * 32 + 2 * e + 1 > r) p1 = 0.f;
-                        }
-                        rowsum += p0 + p1;
-                        hi[e] = pack2<PT>(p0, p1);
-                        if (kSplitP)      // a bf16 is the upper half of an fp32
-                            lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
-                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
-                    }
-                    tmem_st16(sp + c * 16, hi);
-                    if (kSplitP) {
-                        if (c < 3) {
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) lo_hold[c][e] = lo[e];
-                        }
-                        if (c == 2) {            // columns 64..95 have been read
-                            tmem_st16(sp + 64, lo_hold[0]);
-                            tmem_st16(sp + 80, lo_hold[1]);
-                        }
-                        if (c == 3) {            // columns 96..127 have been read
-                            tmem_st16(sp + 96, lo_hold[2]);
-                            tmem_st16(sp + 112, lo);
-                        }
-                    }
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e]), a.sl2, neg_m));
+                    const float p1 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e + 1]), a.sl2, neg_m));
+                    rs[e & 3] += p0 + p1;
+                    hi[e] = pack2<PT>(p0, p1);
+                    if (kSplitP)      // a bf16 is the upper half of an fp32
+                        lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
+                                         p1 - __uint_as_float(hi[e] & 0xffff0000u));
                 }
-            };
-            if (diag) write_p(std::true_type{}); else write_p(std::false_type{});
+                tmem_st16(sp + c * 16, hi);
+                if (kSplitP) tmem_st16(sp + 32 + c * 16, lo);
+            }
             tmem_wait_st();
-            l = fmaf(l, factor, rowsum);
+            l[X] = fmaf(l[X], factor, (rs[0] + rs[1]) + (rs[2] + rs[3]));
             tc_fence_before_sync();
             mbar_arrive(&sh->p_full[X]);
+        };
+        for (int t = 0; t < nt; ++t) {
+            if (t < ntA) do_tile(std::integral_constant<int, 0>{}, t, ntA);
+            if (t < ntB) do_tile(std::integral_constant<int, 1>{}, t, ntB);
         }
-        // ---- epilogue ---------------------------------------------------------------------
-        if (ntX > 0) {
+        // ---- epilogue: each thread normalises and stores its 64 output columns ---------------
+        auto finish = [&](auto Xc, int ntX, int rb) {
+            constexpr int X = decltype(Xc)::value;
+            if (ntX == 0) return;
+            const uint32_t to = tmem_base + X * 2 * kBlk + kBlk + lane_off;
+            const int i = rb * kBlk + r;
+            named_barrier(1 + quarter, 64);                // the partner has read the last row maximum
+            sh->xch[X][half][r] = l[X];
+            named_barrier(1 + quarter, 64);
+            const float lsum = l[X] + sh->xch[X][half ^ 1][r];
             const bool done = wait(&sh->o_done[X], (ntX - 1) & 1);
             tc_fence_after_sync();
-            if (done) {
-                const float inv = 1.f / l;
-                T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h + (int64_t)i * a.st_t;
+            if (!done) return;
+            const float inv = 1.f / lsum;
+            T *orow = static_cast<T *>(a.out) + (int64_t)b * a.st_b + (int64_t)h * a.st_h +
+                      (int64_t)i * a.st_t + half * 64;
 #pragma unroll 1
-                for (int c = 0; c < kD / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(to + c * 32, o);
-                    tmem_wait_ld();
-                    if (i < a.n) {
+            for (int c = 0; c < 2; ++c) {
+                uint32_t o[32];
+                tmem_ld32(to + c * 32, o);
+                tmem_wait_ld();
+                if (i < a.n) {
 #pragma unroll
-                        for (int q4 = 0; q4 < 4; ++q4) {
-                            uint32_t w[4];
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint32_t w[4];
 #pragma unroll
-                            for (int e = 0; e < 4; ++e)
-                                w[e] = pack2<T>(__uint_as_float(o[q4 * 8 + 2 * e]) * inv,
-                                                __uint_as_float(o[q4 * 8 + 2 * e + 1]) * inv);
-                            *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
+                        for (int e = 0; e < 4; ++e)
+                            w[e] = pack2<T>(__uint_as_float(o[q4 * 8 + 2 * e]) * inv,
+                                            __uint_as_float(o[q4 * 8 + 2 * e + 1]) * inv);
+                        *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
-                if (i < a.n) a.lse[(size_t)u * a.n + i] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
-        }
+            if (half == 0 && i < a.n)
+                a.lse[(size_t)u * a.n + i] = (m_used[X] + log2f(lsum)) * 0.6931471805599453f;
+        };
+        finish(std::integral_constant<int, 0>{}, ntA, rbA);
+        finish(std::integral_constant<int, 1>{}, ntB, rbB);
     }
 
     tc_fence_before_sync();
