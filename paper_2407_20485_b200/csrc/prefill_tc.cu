@@ -305,7 +305,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //     S_A(0) S_B(0) | PV_A(0) S_A(1) | PV_B(0) S_B(1) | PV_A(1) S_A(2) | ...
 // so that while one stream's rows are in the softmax warps the other stream's MMAs run.
 //   S = Q K^T        -> TMEM, 128 fp32 columns per stream
-//   softmax warps    : one thread per row.  The running maximum is kept lazily (the accumulator
+//   softmax warps    : two threads per row.  The running maximum is kept lazily (the accumulator
 //                      is rescaled only when the row maximum grows by more than 2^8).  P, rounded
 //                      to the storage type, is written back into the SAME tensor-memory columns
 //                      the logits came from and is read from there as the A operand of the next
@@ -315,8 +315,15 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //   O += P V         -> TMEM, 128 fp32 columns per stream; V is consumed as an MN-major operand
 //                      straight from its TMA tile
 // Tensor memory: S/P_A | O_A | S/P_B | O_B = 512 columns.
-// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-5
-// softmax + epilogue of stream A, warps 6-9 of stream B.
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-9
+// softmax + epilogue: two threads per query row (64 logits each), all eight warps on one
+// stream's tile at a time, the streams taken in turn.
+// Measured on the longest CTA (63 stream tiles, 2393 clocks each against 1440 of tensor work):
+// the softmax warps spend 65 % of their time in the exponential pass at ~12 clocks per logit
+// per scheduler -- the special-function unit issues one warp instruction per 8 clocks and the
+// other ~3.5 instructions per logit do not hide behind it.  Moving part of the exponentials to
+// an FMA-pipe polynomial (+11 instructions each) or the fp16 packing to integer instructions
+// made the pass slower, so neither is used.
 // ============================================================================================
 constexpr int kAttnThreads = 320;
 constexpr int kKStages = 3;                  // K tiles in flight
