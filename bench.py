@@ -212,6 +212,29 @@ def run_ours(args):
                     "flops_per_prefill": U * (w.prefill_flops_per_unit()["pass1"] + 2 * d * rows)}
         del s_ref, sw, kw_
 
+    # ---- separate line: the prompt pruned row by row (n launches of the step kernel) instead of
+    # dense prefill + one selection; a different reading of the method, never part of the headline
+    streamed = None
+    if not args.no_streamed:
+        sc_cache = a2sf.Cache(p, dev)
+        ev_s = torch.empty((n, w.B, w.H), dtype=torch.int32, device=dev)
+        sc_cache.a2sf_prefill_streaming(w.alpha, q, k, v, out=out, evicted=ev_s)      # warm-up
+        es = cuda_events(2)
+        es[0].record()
+        sc_cache.a2sf_prefill_streaming(w.alpha, q, k, v, out=out, evicted=ev_s)
+        es[1].record()
+        torch.cuda.synchronize()
+        ms = es[0].elapsed_time(es[1])
+        # rows 0..M-1 read i slots, the rest M: bytes follow the step's formula with that row count
+        eb = w.elem_bytes
+        row_bytes = sum(U * (2 * min(i, w.budget) * d * eb + 12 * min(i, w.budget) + 6 * d * eb + 16)
+                        for i in range(n))
+        streamed = {"ms_per_prompt": ms, "rows": n, "us_per_row": ms * 1e3 / n,
+                    "gbps": row_bytes / (ms * 1e-3) / 1e9,
+                    "evictions_per_unit": int((ev_s[:, 0, 0] >= 0).sum().item())}
+        sc_cache.close()
+        del ev_s
+
     # ---- end to end through the host-buffer entry points (copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -284,6 +307,7 @@ def run_ours(args):
                      "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
                      "traffic": NCU_DECODE_TRAFFIC.get((w.name, w.B)), "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
         "prefill_zero_weight_rows_skipped": windowed,
+        "prefill_streamed_row_by_row": streamed,
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -480,6 +504,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-streamed", action="store_true",
+                    help="skip the separate timing of the row-by-row streamed prompt")
     ap.add_argument("--no-rotation", action="store_true",
                     help="skip the layer-rotation decode timing of the L2-resident workloads")
     ap.add_argument("--rotation-steps", type=int, default=16, help="decode steps per graph replay")

@@ -231,6 +231,28 @@ int a2sf_decode_step_host(a2sf_cache *cache, float alpha,
                           const void *q_host, const void *k_new_host, const void *v_new_host,
                           void *out_host, int32_t *evicted_slot_host, void *cuda_stream);
 
+/* Empties the cache (count = length = 0, scores 0, positions -1), asynchronously. */
+int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream);
+
+/* ---------------------------------------------------------------------------
+ * Streamed prompt: the cache is pruned WHILE the prompt is processed, row by row, the way
+ * the paper's mask figures (Sec. 3.2, Sec. 4.3) draw it: token i attends only to what
+ * is left of tokens 0..i-1, scores follow Eq. 5 as a recurrence and one token leaves per row
+ * once the budget is full.  This is NOT a2sf_prefill followed by a2sf_cache_load (dense causal
+ * attention, one selection at the end): the two give the same result only while n <= budget.
+ *
+ * Exactly: a2sf_cache_reset, then for i = 0..n-1 the generation step above with
+ * (q_i, k_i, v_i), out_i written to row i of `out`.  Runs as n launches of the step kernel.
+ * q, k, v, out: DEVICE [B][H][n][d] with the strides of a2sf_prefill.  evicted_opt: DEVICE
+ * [n][B][H] int32 (each row as a2sf_decode_step's evicted_slot) or NULL.  On return (the work
+ * is queued on the stream) the cache holds the pruned prompt and generation continues with
+ * a2sf_decode_step.
+ * ------------------------------------------------------------------------- */
+int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n,
+                           const void *q, const void *k, const void *v,
+                           int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                           void *out, int32_t *evicted_opt, void *cuda_stream);
+
 /* Snapshot / restore of the whole cache state into / from caller DEVICE buffers:
  * k, v [B][H][M][d] dtype; scores [B][H][M] fp32; pos [B][H][M] int32; count, len
  * [B][H] int32.  Any pointer may be NULL to skip that part. */

@@ -208,3 +208,23 @@ class Cache:
     def restore(self, snap):
         for k, v in snap.items():
             getattr(self, k)[...] = v
+
+
+def streaming_prefill(Q, K, V, scale: float, alpha, M: int, R: int, force=None, nthreads: int = 1,
+                      lib=None):
+    """The prompt pruned while it is processed, row by row (the reading of the paper's mask
+    figures, Sec. 3.2 / 4.3): starting from an empty cache, token i is one generation step with
+    (q_i, k_i, v_i).  Q, K, V: [U, n, d].  ``force`` [n, U] int32 (or None) overrides the rule's
+    choice per step as in ``Cache.step``.  Returns (out [U,n,d], info [n,U,3], scores [n,U,3],
+    cache)."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    U, n, d = Q.shape
+    cache = Cache(U, d, M, R, scale, lib=lib)
+    out = np.empty((U, n, d), dtype=np.float64)
+    info = np.empty((n, U, 3), dtype=np.int32)
+    sc = np.empty((n, U, 3), dtype=np.float64)
+    for i in range(n):
+        o, info[i], sc[i] = cache.step(Q[:, i], K[:, i], V[:, i], alpha,
+                                        force=None if force is None else force[i], nthreads=nthreads)
+        out[:, i] = o
+    return out, info, sc, cache

@@ -63,6 +63,8 @@ def _load():
         "a2sf_cache_load": (ctypes.c_int, [vp, i32, vp, vp, i64, i64, i64, vp, vp, vp]),
         "a2sf_decode_step": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_decode_step_host": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
+        "a2sf_cache_reset": (ctypes.c_int, [vp, vp]),
+        "a2sf_prefill_streaming": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp]),
         "a2sf_cache_export": (ctypes.c_int, [vp] * 8),
         "a2sf_cache_import": (ctypes.c_int, [vp] * 8),
         "a2sf_kernel_launch_count": (ctypes.c_int64, []),
@@ -262,6 +264,27 @@ class Cache:
         _check(lib.a2sf_decode_step_host(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),
                                          _ptr(out), _ptr(evicted), _stream(stream)),
                "a2sf_decode_step_host")
+
+    def a2sf_cache_reset(self, stream=None):
+        _check(lib.a2sf_cache_reset(self.handle, _stream(stream)), "a2sf_cache_reset")
+
+    def a2sf_prefill_streaming(self, alpha, q, k, v, out=None, evicted=None, stream=None):
+        """Prunes while the prompt is processed: q, k, v [B,H,n,d] (one stride set).  Returns
+        (out [B,H,n,d], evicted [n,B,H] int32)."""
+        B, H, n, d = q.shape
+        assert (B, H, d) == (self.p.B, self.p.H, self.d) and q.dtype == self.torch_dtype
+        assert k.shape == q.shape and v.shape == q.shape
+        assert _strides(k) == _strides(q) and _strides(v) == _strides(q)
+        if out is None:
+            out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+        assert _strides(out) == _strides(q)
+        if evicted is None:
+            evicted = torch.empty((n, B, H), dtype=torch.int32, device=q.device)
+        sb, sh, st = _strides(q)
+        _check(lib.a2sf_prefill_streaming(self.handle, alpha, n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st,
+                                          _ptr(out), _ptr(evicted), _stream(stream)),
+               "a2sf_prefill_streaming")
+        return out, evicted
 
     def state_tensors(self, device=None):
         device = device or self.mem.device

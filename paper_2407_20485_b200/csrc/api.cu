@@ -301,6 +301,7 @@ int a2sf_cache_create(const a2sf_params *p, void *device_mem, size_t bytes, a2sf
     c->view.sched = reinterpret_cast<int32_t *>(b + L.sched);
     c->view.U = p->B * p->H; c->view.M = p->budget; c->view.R = p->recent;
     c->view.d = p->d; c->view.dtype = p->dtype; c->view.scale = eff_scale(p);
+    c->view.io_H = p->H; c->view.io_st_b = (long long)p->H * p->d; c->view.io_st_h = p->d;
     c->st_q = b + L.st_q; c->st_k = b + L.st_k; c->st_v = b + L.st_v; c->st_out = b + L.st_out;
     c->st_ev = reinterpret_cast<int32_t *>(b + L.st_ev);
     // empty cache: zero scores and counters, positions -1
@@ -348,6 +349,48 @@ int a2sf_decode_step(a2sf_cache *cache, float alpha, const void *q, const void *
     if (launch_decode_step(cache->view, alpha, nullptr, q, k_new, v_new, out, evicted_slot,
                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream)
+{
+    if (!cache) return A2SF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const CacheView &c = cache->view;
+    const size_t U = c.U, M = c.M;
+    if (cudaMemsetAsync(c.S, 0, U * M * 4, s) != cudaSuccess ||
+        cudaMemsetAsync(c.pos, 0xff, U * M * 4, s) != cudaSuccess ||
+        cudaMemsetAsync(c.count, 0, U * 4, s) != cudaSuccess ||
+        cudaMemsetAsync(c.len, 0, U * 4, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n, const void *q, const void *k,
+                           const void *v, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                           void *out, int32_t *evicted_opt, void *cuda_stream)
+{
+    if (!cache || n < 1 || !q || !k || !v || !out) return A2SF_ERR_INVALID_ARG;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
+    int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
+    if (rc != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16))
+        return A2SF_ERR_INVALID_ARG;
+    rc = a2sf_cache_reset(cache, cuda_stream);
+    if (rc != A2SF_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    CacheView view = cache->view;
+    view.io_st_b = stride_b;
+    view.io_st_h = stride_h;
+    const size_t eb = elem_bytes(cache->p.dtype), U = view.U;
+    for (int32_t i = 0; i < n; ++i) {
+        const size_t off = (size_t)i * (size_t)stride_t * eb;
+        int32_t *ev = evicted_opt ? evicted_opt + (size_t)i * U : cache->st_ev;
+        if (launch_decode_step(view, alpha, nullptr, static_cast<const char *>(q) + off,
+                               static_cast<const char *>(k) + off, static_cast<const char *>(v) + off,
+                               static_cast<char *>(out) + off, ev, s) != cudaSuccess)
+            return A2SF_ERR_CUDA;
+    }
     return A2SF_OK;
 }
 

@@ -133,7 +133,17 @@ struct CacheView {
     int32_t *sched;       // [2] unit-claim counter and finished-CTA counter of the decode kernel
     int U, M, R, d, dtype;
     float scale;
+    // where unit u = b*io_H + h finds its row of the step's q, k_new, v_new and out (elements):
+    // [B][H][d] contiguous for a generation step, a token's rows of a [B][H][n][d] tensor when
+    // the prompt is streamed through the step kernel
+    int io_H;
+    long long io_st_b, io_st_h;
 };
+
+__host__ __device__ __forceinline__ size_t io_offset(const CacheView &c, int u)
+{
+    return (size_t)(u / c.io_H) * (size_t)c.io_st_b + (size_t)(u % c.io_H) * (size_t)c.io_st_h;
+}
 
 cudaError_t launch_cache_load(const CacheView &c, int H, int n, const void *k, const void *v,
                               Strides st, const float *scores, const int32_t *kept,

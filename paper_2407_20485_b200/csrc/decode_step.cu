@@ -104,6 +104,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     __shared__ int s_target;
 
     const int u = blockIdx.x / C;
+    const size_t uo = io_offset(c, u);           // this unit's row of q, k_new, v_new, out
     const float alpha = unit_alpha(alpha_vec, u, alpha_all);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int sub = lane % LPR, rsel = lane / LPR;
@@ -121,7 +122,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     int32_t *posu = c.pos + (size_t)u * M;
 
     float qf[VEC];
-    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
+    Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + uo + sub * VEC), qf);
 
     // ---- (i) logits of the slice, and (rank 0) of the new key ---------------------------------
     const int ngroups = (nloc + RPW - 1) / RPW;
@@ -148,7 +149,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     }
     if (warp == 0 && rank == 0) {
         float kf[VEC];
-        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC), kf);
+        Elem<T>::unpack(*reinterpret_cast<const uint4 *>(k_new + uo + sub * VEC), kf);
         float dot = 0.f;
 #pragma unroll
         for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
@@ -204,7 +205,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         float o = 0.f;
 #pragma unroll
         for (int x = 0; x < NW; ++x) o += part[x * D + tid];
-        if (rank == 0) o = fmaf(w[nloc], Elem<T>::to_float(v_new[(size_t)u * D + tid]), o);
+        if (rank == 0) o = fmaf(w[nloc], Elem<T>::to_float(v_new[uo + tid]), o);
         xch.out[tid] = o;
     }
     if (tid == 0) { xch.m = m_loc; xch.l = l_loc; }
@@ -224,7 +225,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
             const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
             o = fmaf(x->out[tid], expf(x->m - m), o);
         }
-        out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
+        out[uo + tid] = Elem<T>::from_float(o / l);
     }
 
     // ---- (iv) S <- alpha*S + a for the slice ; local eviction candidate ---------------------------
@@ -286,10 +287,10 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         if (target >= 0) {
             if (tid < LPR)
                 *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
-                    *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
+                    *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
             else if (tid < 2 * LPR)
                 *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
-                    *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
+                    *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
         }
         if (tid == 0) {
             if (target >= 0) {
@@ -503,6 +504,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             if (lane == 0) tc::mbar_arrive(&sh->uq_empty[qi]);
             const int p = c.len[u];
             const float alpha = unit_alpha(alpha_vec, u, alpha_all);
+            const size_t uo = io_offset(c, u);   // this unit's row of q, k_new, v_new, out
             T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
             T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
             float *Su = c.S + (size_t)u * M;
@@ -511,9 +513,9 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             // every global word this unit needs is requested up front, so its latency hides
             // behind the K and V phases instead of stalling the reductions and the epilogue
             float qf[VEC];
-            Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + (size_t)u * D + sub * VEC), qf);
-            const uint4 knew_raw = *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + sub * VEC);
-            const float vnew_val = tid < D ? Elem<T>::to_float(v_new[(size_t)u * D + tid]) : 0.f;
+            Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + uo + sub * VEC), qf);
+            const uint4 knew_raw = *reinterpret_cast<const uint4 *>(k_new + uo + sub * VEC);
+            const float vnew_val = tid < D ? Elem<T>::to_float(v_new[uo + tid]) : 0.f;
             float s_pre[kPrefetchSlots];
             int pos_pre[kPrefetchSlots];
 #pragma unroll
@@ -615,7 +617,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
 #pragma unroll
                 for (int x = 0; x < NW; ++x) o += part[x * D + tid];
                 o = fmaf(e_self, vnew_val, o);
-                out[(size_t)u * D + tid] = Elem<T>::from_float(o / l);
+                out[uo + tid] = Elem<T>::from_float(o / l);
             }
 
             // (iv) S <- alpha*S + a ; (v) argmin over the non-recent slots
@@ -658,10 +660,10 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             if (target >= 0) {
                 if (tid < LPR)
                     *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
-                        *reinterpret_cast<const uint4 *>(k_new + (size_t)u * D + tid * VEC);
+                        *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
                 else if (tid < 2 * LPR)
                     *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
-                        *reinterpret_cast<const uint4 *>(v_new + (size_t)u * D + (tid - LPR) * VEC);
+                        *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
             }
             if (tid == 0 && !*abort_flag) {
                 if (target >= 0) {

@@ -412,3 +412,73 @@ def test_per_unit_alpha_equals_unit_by_unit_scalar_steps():
             np.testing.assert_array_equal(info[u], i1[0])
             np.testing.assert_array_equal(a.S[u], singles[u].S[0])
             np.testing.assert_array_equal(a.pos[u], singles[u].pos[0])
+
+
+# ---- prompt pruned row by row (streamed prefill) ------------------------------------------------
+def test_streamed_prompt_without_eviction_is_the_dense_prefill():
+    """While the budget holds the whole prompt nothing is evicted, so processing it token by
+    token must reproduce dense causal attention (Eq. 3) and the scores of Eq. 5."""
+    rng = np.random.default_rng(21)
+    n, d, alpha = 23, 8, 0.7
+    Q, K, V = _rand_unit(rng, n, d)
+    out, info, _, cache = oracle.streaming_prefill(Q[None], K[None], V[None], 0.35, alpha, M=n, R=5)
+    P = _brute_probs(Q, K, 0.35)
+    np.testing.assert_allclose(out[0], P @ V, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(cache.S[0], _brute_scores(P, alpha), rtol=1e-12, atol=1e-15)
+    np.testing.assert_array_equal(cache.pos[0], np.arange(n))
+    assert (info[:, 0, 0] == -1).all() and cache.count[0] == n and cache.len[0] == n
+
+
+def test_streamed_prompt_with_recent_equal_budget_is_a_sliding_window():
+    """R = M: every step drops the oldest token, so row i sees tokens i-M .. i only."""
+    rng = np.random.default_rng(22)
+    n, d, M = 30, 4, 6
+    Q, K, V = _rand_unit(rng, n, d)
+    out, _, _, _ = oracle.streaming_prefill(Q[None], K[None], V[None], 0.5, 0.4, M=M, R=M)
+    for i in range(n):
+        lo = max(0, i - M)
+        s = (K[lo:i + 1] @ Q[i]) * 0.5
+        w = np.exp(s - s.max())
+        np.testing.assert_allclose(out[0, i], (w / w.sum()) @ V[lo:i + 1], rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("M,R,alpha", [(6, 2, 0.5), (5, 0, 0.8), (7, 3, 1.0), (4, 1, 0.0)])
+def test_streamed_prompt_matches_a_mask_matrix_construction(M, R, alpha):
+    """The same policy written the way the paper draws it: an n x n mask built row by row over
+    full-length score vectors (no slots, no cache object)."""
+    rng = np.random.default_rng(23 + M)
+    n, d, scale = 26, 6, 0.4
+    Q, K, V = _rand_unit(rng, n, d)
+    out, info, _, cache = oracle.streaming_prefill(Q[None], K[None], V[None], scale, alpha, M=M, R=R)
+    alive = np.zeros(n, dtype=bool)
+    S = np.zeros(n)
+    for i in range(n):
+        alive[i] = True
+        idx = np.flatnonzero(alive)
+        s = (K[idx] @ Q[i]) * scale
+        w = np.exp(s - s.max())
+        w /= w.sum()
+        np.testing.assert_allclose(out[0, i], w @ V[idx], rtol=1e-11, atol=1e-12)
+        S *= alpha
+        S[idx] += w
+        if alive.sum() > M:
+            cand = [j for j in idx if j <= i - R]              # outside the recent window
+            victim = min(cand, key=lambda j: (S[j], j))
+            alive[victim] = False
+            S[victim] = 0.0
+    kept = np.sort(cache.pos[0, :cache.count[0]])
+    np.testing.assert_array_equal(kept, np.flatnonzero(alive))
+    order = np.argsort(cache.pos[0, :cache.count[0]])
+    np.testing.assert_allclose(cache.S[0, :cache.count[0]][order], S[alive], rtol=1e-11, atol=1e-14)
+
+
+def test_streamed_prompt_differs_from_one_shot_selection():
+    """With a budget below the prompt length the two readings part: a token evicted early cannot
+    be attended to later, so outputs of late rows differ from dense attention."""
+    rng = np.random.default_rng(29)
+    n, d = 40, 8
+    Q, K, V = _rand_unit(rng, n, d)
+    out, _, _, _ = oracle.streaming_prefill(Q[None], K[None], V[None], 0.35, 0.5, M=8, R=4)
+    dense = _brute_probs(Q, K, 0.35) @ V
+    np.testing.assert_allclose(out[0, :9], dense[:9], rtol=1e-12, atol=1e-13)   # nothing evicted yet
+    assert np.abs(out[0, 20:] - dense[20:]).max() > 1e-3

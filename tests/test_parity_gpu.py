@@ -241,6 +241,74 @@ def test_decode_steps_replayed_from_a_cuda_graph_match_direct_launches(name, kw)
     assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
 
 
+# ---- prompt pruned while it is processed (row by row) ------------------------------------------
+@pytest.mark.parametrize("name,kw", [
+    ("tiny_fp32", dict()),                                                     # fp32, d = 64
+    ("llama2_7b", dict(H=5, n=333, budget=64, recent=32)),                     # bf16 streaming kernel
+    ("opt_6p7b", dict(B=2, H=3, n=260, budget=48, recent=0)),                  # fp16, all selective
+    ("llama2_13b", dict(B=1, H=2, n=100, budget=128, recent=64)),              # budget never reached
+    ("long_context", dict(H=2, n=700, budget=512, recent=256)),                # cluster split-K
+    ("llama2_7b", dict(H=3, n=150, budget=32, recent=32)),                     # sliding window
+])
+def test_streamed_prompt_against_the_oracle(name, kw):
+    import oracle
+    from parity_util import ParityReport, TIE_RTOL, check_out, check_scores, to_f64
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    cache = a2sf.Cache(p)
+    q2 = q[:, :, 5:6].contiguous()
+    cache.a2sf_decode_step(w.alpha, q2[:, :, 0], q2[:, :, 0], q2[:, :, 0],
+                           torch.empty_like(q2[:, :, 0]),
+                           torch.empty((w.B, w.H), dtype=torch.int32, device="cuda"))   # dirty the cache
+    out, ev = cache.a2sf_prefill_streaming(w.alpha, q, k, v)
+    torch.cuda.synchronize()
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+    U, n = w.units, w.n
+    ev_g = ev.cpu().numpy().reshape(n, U)
+    force = np.where(ev_g == -1, -3, ev_g).astype(np.int32)
+    Q, K, V = (to_f64(t).reshape(U, n, w.d) for t in (q, k, v))
+    o_out, info, sc, oc = oracle.streaming_prefill(Q, K, V, w.scale, w.alpha, w.budget, w.recent,
+                                                   force=force, nthreads=oracle.host_threads())
+    rep = ParityReport()
+    excused = evictions = 0
+    for i in range(n):
+        for u in range(U):
+            if info[i, u, 1] == -1:
+                assert ev_g[i, u] == -1, f"row {i} unit {u}: cache not full but evicted {ev_g[i, u]}"
+                continue
+            evictions += 1
+            assert ev_g[i, u] != -1
+            if ev_g[i, u] != info[i, u, 1]:
+                a_, b_ = sc[i, u, 0], sc[i, u, 1]
+                assert abs(a_ - b_) <= TIE_RTOL * max(abs(a_), abs(b_)), (
+                    f"row {i} unit {u}: evicted {ev_g[i, u]} (score {a_!r}), rule picks "
+                    f"{info[i, u, 1]} (score {b_!r})")
+                excused += 1
+    assert excused <= max(2, evictions // 200)
+    if w.budget < n:
+        assert evictions == U * (n - w.budget)
+    check_out(to_f64(out).reshape(U, n, w.d), o_out, w.dtype, rep, "streamed out")
+    st = cache.a2sf_cache_export()
+    torch.cuda.synchronize()
+    cnt = st["count"].cpu().numpy().reshape(U)
+    np.testing.assert_array_equal(cnt, oc.count)
+    np.testing.assert_array_equal(st["len"].cpu().numpy().reshape(U), oc.len)
+    pos = st["pos"].cpu().numpy().reshape(U, -1)
+    S = to_f64(st["scores"]).reshape(U, -1)
+    Kc = to_f64(st["k"]).reshape(U, w.budget, w.d)
+    for u in range(U):
+        c = int(cnt[u])
+        np.testing.assert_array_equal(pos[u, :c], oc.pos[u, :c])
+        check_scores(S[u, :c], oc.S[u, :c], rep, "streamed cache scores")
+        assert np.array_equal(Kc[u, :c], oc.K[u, :c])
+    print(f"\n[streamed] {w.name}: units={U} n={n} M={w.budget} R={w.recent} evictions={evictions} "
+          f"excused={excused} max_out={rep.max_out_err:.3g} max_score_rel={rep.max_score_rel:.3g}")
+    cache.close()
+
+
 # ---- scoring pass that leaves out rows whose forgetting weight is exactly zero ------------------
 @pytest.mark.parametrize("name,kw,alphas", [
     ("llama2_13b", dict(B=1, H=3, n=1100), [0.5, 0.9, 0.0, 1.0, 0.3]),      # tensor-core pass
