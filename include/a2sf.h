@@ -61,6 +61,7 @@ typedef struct a2sf_params {
     float alpha;
     float scale;
     int32_t flags;               /* 0 or A2SF_FLAG_* */
+    int32_t score_window;        /* 0, or W > 0: see a2sf_score_window_bound */
 } a2sf_params;
 
 /* Scoring pass: Eq. 5 weighs query row i with alpha^(n-1-i).  Once that weight is below
@@ -68,6 +69,15 @@ typedef struct a2sf_params {
  * pass leaves those rows out: O(n * window) instead of O(n^2) work with bit-identical scores.
  * Off by default; alpha = 1 has no such rows. */
 #define A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS 1
+
+/* Truncated scoring pass.  With score_window = W > 0 the sum of Eq. 5 runs over the last W
+ * query rows only, S_j = sum_{i >= max(j, n-W)} alpha^(n-1-i) P_ij: O(n * W) work.  Every
+ * probability is at most 1, so each score falls short of the full sum by at most
+ *     sum_{a=W}^{n-1} alpha^a = alpha^W (1 - alpha^(n-W)) / (1 - alpha)      (n - W for alpha = 1),
+ * which this function returns (0 when W = 0 or W >= n).  The attention output and lse are not
+ * affected.  Unlike A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS this changes the scores: the kept set may
+ * differ wherever two scores are closer than the bound. */
+double a2sf_score_window_bound(float alpha, int32_t n, int32_t score_window);
 
 typedef struct a2sf_cache a2sf_cache;   /* opaque, owned by the library */
 
@@ -231,6 +241,16 @@ int a2sf_decode_step_host(a2sf_cache *cache, float alpha,
                           const void *q_host, const void *k_new_host, const void *v_new_host,
                           void *out_host, int32_t *evicted_slot_host, void *cuda_stream);
 
+/* Several tokens appended in one call (a draft that was accepted, a prompt continued in
+ * chunks): exactly `steps` generation steps in order, token t taking row t of q, k_new,
+ * v_new and writing row t of out -- DEVICE [B][H][steps][d] with element strides as in
+ * a2sf_prefill.  evicted_opt: DEVICE [steps][B][H] int32 or NULL.  Runs as `steps` launches;
+ * the result is bit-identical to calling a2sf_decode_step `steps` times. */
+int a2sf_decode_multi(a2sf_cache *cache, float alpha, int32_t steps,
+                      const void *q, const void *k_new, const void *v_new,
+                      int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                      void *out, int32_t *evicted_opt, void *cuda_stream);
+
 /* Empties the cache (count = length = 0, scores 0, positions -1), asynchronously. */
 int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream);
 
@@ -241,8 +261,8 @@ int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream);
  * once the budget is full.  This is NOT a2sf_prefill followed by a2sf_cache_load (dense causal
  * attention, one selection at the end): the two give the same result only while n <= budget.
  *
- * Exactly: a2sf_cache_reset, then for i = 0..n-1 the generation step above with
- * (q_i, k_i, v_i), out_i written to row i of `out`.  Runs as n launches of the step kernel.
+ * Exactly: a2sf_cache_reset, then a2sf_decode_multi over the n prompt tokens (the generation
+ * step with (q_i, k_i, v_i), out_i written to row i of `out`): n launches of the step kernel.
  * q, k, v, out: DEVICE [B][H][n][d] with the strides of a2sf_prefill.  evicted_opt: DEVICE
  * [n][B][H] int32 (each row as a2sf_decode_step's evicted_slot) or NULL.  On return (the work
  * is queued on the stream) the cache holds the pruned prompt and generation continues with

@@ -25,7 +25,8 @@ A2SF_ERR_TIMEOUT, A2SF_ERR_WORKSPACE = -4, -5
 class a2sf_params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32),
                 ("dtype", ctypes.c_int32), ("budget", ctypes.c_int32), ("recent", ctypes.c_int32),
-                ("alpha", ctypes.c_float), ("scale", ctypes.c_float), ("flags", ctypes.c_int32)]
+                ("alpha", ctypes.c_float), ("scale", ctypes.c_float), ("flags", ctypes.c_int32),
+                ("score_window", ctypes.c_int32)]
 
 
 class A2SFError(RuntimeError):
@@ -64,6 +65,8 @@ def _load():
         "a2sf_decode_step": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_decode_step_host": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_cache_reset": (ctypes.c_int, [vp, vp]),
+        "a2sf_score_window_bound": (ctypes.c_double, [f32, i32, i32]),
+        "a2sf_decode_multi": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp]),
         "a2sf_prefill_streaming": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp]),
         "a2sf_cache_export": (ctypes.c_int, [vp] * 8),
         "a2sf_cache_import": (ctypes.c_int, [vp] * 8),
@@ -107,8 +110,12 @@ A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS = 1
 
 
 def make_params(B: int, H: int, d: int, dtype: torch.dtype, budget: int, recent: int,
-                alpha: float, scale: float = 0.0, flags: int = 0) -> a2sf_params:
-    return a2sf_params(B, H, d, _DTYPE_CODE[dtype], budget, recent, alpha, scale, flags)
+                alpha: float, scale: float = 0.0, flags: int = 0, score_window: int = 0) -> a2sf_params:
+    return a2sf_params(B, H, d, _DTYPE_CODE[dtype], budget, recent, alpha, scale, flags, score_window)
+
+
+def a2sf_score_window_bound(alpha: float, n: int, score_window: int) -> float:
+    return float(lib.a2sf_score_window_bound(alpha, n, score_window))
 
 
 def a2sf_kernel_launch_count() -> int:
@@ -268,9 +275,18 @@ class Cache:
     def a2sf_cache_reset(self, stream=None):
         _check(lib.a2sf_cache_reset(self.handle, _stream(stream)), "a2sf_cache_reset")
 
+    def a2sf_decode_multi(self, alpha, q, k_new, v_new, out=None, evicted=None, stream=None):
+        """Appends the tokens of q, k_new, v_new [B,H,steps,d] one after the other."""
+        return self._token_rows(lib.a2sf_decode_multi, "a2sf_decode_multi", alpha, q, k_new, v_new,
+                                out, evicted, stream)
+
     def a2sf_prefill_streaming(self, alpha, q, k, v, out=None, evicted=None, stream=None):
         """Prunes while the prompt is processed: q, k, v [B,H,n,d] (one stride set).  Returns
         (out [B,H,n,d], evicted [n,B,H] int32)."""
+        return self._token_rows(lib.a2sf_prefill_streaming, "a2sf_prefill_streaming", alpha, q, k, v,
+                                out, evicted, stream)
+
+    def _token_rows(self, fn, name, alpha, q, k, v, out, evicted, stream):
         B, H, n, d = q.shape
         assert (B, H, d) == (self.p.B, self.p.H, self.d) and q.dtype == self.torch_dtype
         assert k.shape == q.shape and v.shape == q.shape
@@ -281,9 +297,8 @@ class Cache:
         if evicted is None:
             evicted = torch.empty((n, B, H), dtype=torch.int32, device=q.device)
         sb, sh, st = _strides(q)
-        _check(lib.a2sf_prefill_streaming(self.handle, alpha, n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st,
-                                          _ptr(out), _ptr(evicted), _stream(stream)),
-               "a2sf_prefill_streaming")
+        _check(fn(self.handle, alpha, n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st,
+                  _ptr(out), _ptr(evicted), _stream(stream)), name)
         return out, evicted
 
     def state_tensors(self, device=None):

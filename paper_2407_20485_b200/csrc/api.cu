@@ -28,6 +28,7 @@ static int check_params(const a2sf_params *p)
     if (p->d != 64 && p->d != 128) return A2SF_ERR_UNSUPPORTED;
     if ((int64_t)p->B * p->H > 0x7fffffff) return A2SF_ERR_INVALID_ARG;
     if (p->flags & ~A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) return A2SF_ERR_INVALID_ARG;
+    if (p->score_window < 0) return A2SF_ERR_INVALID_ARG;
     return A2SF_OK;
 }
 
@@ -115,6 +116,7 @@ static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
+    a.window_rows = p->score_window;
     a.v_half = nullptr; a.v_flag = nullptr;
     if (prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d) > 0) {
         char *extra = static_cast<char *>(workspace) + align_up((size_t)p->B * p->H * n * sizeof(float));
@@ -165,6 +167,7 @@ static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
+    a.window_rows = p->score_window;
     a.v_half = nullptr; a.v_flag = nullptr;
     return run_scores_and_select(p, n, a, kept_idx, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -352,6 +355,14 @@ int a2sf_decode_step(a2sf_cache *cache, float alpha, const void *q, const void *
     return A2SF_OK;
 }
 
+double a2sf_score_window_bound(float alpha, int32_t n, int32_t score_window)
+{
+    if (score_window <= 0 || score_window >= n || !(alpha >= 0.f && alpha <= 1.f)) return 0.0;
+    const double a = alpha;
+    if (a >= 1.0) return (double)(n - score_window);
+    return std::pow(a, (double)score_window) * (1.0 - std::pow(a, (double)(n - score_window))) / (1.0 - a);
+}
+
 int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream)
 {
     if (!cache) return A2SF_ERR_INVALID_ARG;
@@ -363,6 +374,33 @@ int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream)
         cudaMemsetAsync(c.count, 0, U * 4, s) != cudaSuccess ||
         cudaMemsetAsync(c.len, 0, U * 4, s) != cudaSuccess)
         return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_decode_multi(a2sf_cache *cache, float alpha, int32_t steps, const void *q, const void *k_new,
+                      const void *v_new, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                      void *out, int32_t *evicted_opt, void *cuda_stream)
+{
+    if (!cache || steps < 1 || !q || !k_new || !v_new || !out) return A2SF_ERR_INVALID_ARG;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
+    int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
+    if (rc != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16))
+        return A2SF_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    CacheView view = cache->view;
+    view.io_st_b = stride_b;
+    view.io_st_h = stride_h;
+    const size_t eb = elem_bytes(cache->p.dtype), U = view.U;
+    for (int32_t i = 0; i < steps; ++i) {
+        const size_t off = (size_t)i * (size_t)stride_t * eb;
+        int32_t *ev = evicted_opt ? evicted_opt + (size_t)i * U : cache->st_ev;
+        if (launch_decode_step(view, alpha, nullptr, static_cast<const char *>(q) + off,
+                               static_cast<const char *>(k_new) + off,
+                               static_cast<const char *>(v_new) + off,
+                               static_cast<char *>(out) + off, ev, s) != cudaSuccess)
+            return A2SF_ERR_CUDA;
+    }
     return A2SF_OK;
 }
 
@@ -378,20 +416,8 @@ int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n, const void
         return A2SF_ERR_INVALID_ARG;
     rc = a2sf_cache_reset(cache, cuda_stream);
     if (rc != A2SF_OK) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    CacheView view = cache->view;
-    view.io_st_b = stride_b;
-    view.io_st_h = stride_h;
-    const size_t eb = elem_bytes(cache->p.dtype), U = view.U;
-    for (int32_t i = 0; i < n; ++i) {
-        const size_t off = (size_t)i * (size_t)stride_t * eb;
-        int32_t *ev = evicted_opt ? evicted_opt + (size_t)i * U : cache->st_ev;
-        if (launch_decode_step(view, alpha, nullptr, static_cast<const char *>(q) + off,
-                               static_cast<const char *>(k) + off, static_cast<const char *>(v) + off,
-                               static_cast<char *>(out) + off, ev, s) != cudaSuccess)
-            return A2SF_ERR_CUDA;
-    }
-    return A2SF_OK;
+    return a2sf_decode_multi(cache, alpha, n, q, k, v, stride_b, stride_h, stride_t, out, evicted_opt,
+                             cuda_stream);
 }
 
 int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas, const void *q,

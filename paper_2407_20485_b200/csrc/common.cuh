@@ -107,6 +107,7 @@ struct PrefillArgs {
     float scale, alpha;
     const float *alpha_vec;   // per-unit forgetting factors [U] on the device, or nullptr (use alpha)
     int skip_zero_rows;       // scoring pass: leave out rows whose weight is exactly 0 in fp32
+    int window_rows;          // scoring pass: only the last window_rows query rows (0 = all)
     void *v_half;             // bf16 tensor-core path: fp16 copy of V, contiguous [U][n][d] (workspace)
     int *v_flag;              // ... and the word that says the copy is not exact (workspace)
 };

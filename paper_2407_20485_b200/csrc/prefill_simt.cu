@@ -177,14 +177,17 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
         const int i_min = span >= (float)a.n ? 0 : min(a.n - 1, a.n - (int)span);
         i_first = max(i_first, (i_min / kTile) * kTile);
     }
+    // truncated sum: only the last window_rows query rows enter (the caller accepts the bound)
+    const int i_window = a.window_rows > 0 ? max(0, a.n - a.window_rows) : 0;
+    i_first = max(i_first, (i_window / kTile) * kTile);
     float acc = 0.f;
     for (int i0 = i_first; i0 < a.n; i0 += kTile) {
         __syncthreads();
         load_tile<T, D>(Qs, Q, a.st.t, i0, a.n);
         if (threadIdx.x < kTile) {
             const int i = i0 + threadIdx.x;
-            float cv = INFINITY;                     // rows past n contribute nothing
-            if (i < a.n) {
+            float cv = INFINITY;                     // rows past n or before the window: nothing
+            if (i < a.n && i >= i_window) {
                 const int age = a.n - 1 - i;
                 cv = lse[i] * kLog2e + (age == 0 ? 0.f : (float)age * neg_log2_alpha);
             }

@@ -84,6 +84,7 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
     a.alpha = p->alpha;
     a.alpha_vec = nullptr;
     a.skip_zero_rows = 0;
+    a.window_rows = 0;
     a.v_half = nullptr;
     a.v_flag = nullptr;
     if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;

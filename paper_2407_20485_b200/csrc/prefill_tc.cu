@@ -46,6 +46,7 @@ struct ScoreArgs {
     float alpha;          // forgetting factor, or per unit:
     const float *alpha_vec;
     int skip_zero_rows;   // leave out query tiles whose forgetting weight underflows to exactly 0
+    int window_rows;      // only the last window_rows query rows enter the sum (0 = all)
 };
 
 struct ScoreShared {
@@ -149,6 +150,9 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         const int i_min = span >= (float)a.n ? 0 : min(a.n - 1, a.n - (int)span);
         t_first = max(kb, i_min / kBlk);
     }
+    // truncated sum: rows before n - window_rows are left out (their constants become +inf)
+    const int i_window = a.window_rows > 0 ? max(0, a.n - a.window_rows) : 0;
+    t_first = max(t_first, i_window / kBlk);
     const int ntiles = ntile_total - t_first;          // query-row tiles t_first .. last
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int *abort_flag = &sh->abort_flag;
@@ -197,7 +201,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             for (int e = 0; e < 4; ++e) {
                 const int i = i0 + lane * 4 + e;
                 const int age = a.n - 1 - i;
-                c4[e] = i < a.n ? fmaf(__ldg(lse + i), kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha)
+                c4[e] = (i < a.n && i >= i_window) ? fmaf(__ldg(lse + i), kLog2e, age == 0 ? 0.f : (float)age * neg_log2_alpha)
                                 : INFINITY;
             }
             int ok = 1;
@@ -850,6 +854,7 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     sa.alpha = a.alpha;
     sa.alpha_vec = a.alpha_vec;
     sa.skip_zero_rows = a.skip_zero_rows;
+    sa.window_rows = a.window_rows;
     const dim3 grid((unsigned)((size_t)a.B * a.H * ((a.n + kBlk - 1) / kBlk)));
     score_pass_tc<<<grid, kScoreThreads, kScoreSmemBytes, s>>>(mq, mk, sa, dtype == A2SF_BF16 ? 1 : 0);
     count_launch();

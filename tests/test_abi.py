@@ -2,6 +2,8 @@
 rejects bad arguments on the host before anything is launched."""
 import ctypes
 import re
+
+import numpy as np
 from pathlib import Path
 
 import pytest
@@ -109,3 +111,16 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     monkeypatch.setattr(binding, "_LIB_PATH", tmp_path / "liba2sf.so")
     with pytest.raises(ImportError, match="no CPU fallback"):
         binding._load()
+
+
+def test_score_window_bound_is_the_tail_of_the_geometric_series():
+    """Host arithmetic only: the bound equals the summed weights of the rows left out."""
+    from paper_2407_20485_b200 import binding as a2sf
+
+    for alpha, n, Wn in [(0.5, 100, 10), (0.9, 4096, 200), (1.0, 50, 20), (0.0, 30, 3), (0.3, 10, 10),
+                         (0.7, 10, 0), (0.99, 500, 499)]:
+        # fp32 alpha, as the library receives it
+        a = float(np.float32(alpha))
+        tail = sum(a ** age for age in range(Wn, n)) if 0 < Wn < n else 0.0
+        got = a2sf.a2sf_score_window_bound(alpha, n, Wn)
+        assert abs(got - tail) <= 1e-12 * max(1.0, tail), (alpha, n, Wn, got, tail)

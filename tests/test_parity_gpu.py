@@ -195,6 +195,45 @@ def test_export_import_round_trip_and_generator_on_device():
     assert a2sf.a2sf_kernel_launch_count() > 0
 
 
+# ---- truncated scoring pass: only the last W query rows, with a stated bound -------------------
+@pytest.mark.parametrize("name,kw,windows", [
+    ("llama2_13b", dict(B=1, H=3, n=1100, alpha=0.9), [1, 100, 128, 300, 1100, 5000]),   # tensor-core pass
+    ("tiny_fp32", dict(n=333, budget=64, recent=32, alpha=0.8), [7, 64, 200]),            # CUDA-core pass
+])
+def test_truncated_scoring_window_matches_partial_sum_and_respects_bound(name, kw, windows):
+    import oracle
+    from parity_util import ParityReport, check_scores, to_f64
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    p0 = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    out0, S0, kept0, lse0 = a2sf.a2sf_prefill(p0, q, k, v)
+    U, n = w.units, w.n
+    Q, K, V = (to_f64(t).reshape(U, n, w.d) for t in (q, k, v))
+    rep = ParityReport()
+    for Wn in windows:
+        pw = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha, score_window=Wn)
+        out1, S1, kept1, lse1 = a2sf.a2sf_prefill(pw, q, k, v)
+        S2, kept2 = a2sf.a2sf_rescore(pw, q, k, lse0)
+        torch.cuda.synchronize()
+        assert torch.equal(out1, out0) and torch.equal(lse1, lse0)       # attention itself is untouched
+        assert torch.equal(S1, S2) and torch.equal(kept1, kept2)
+        i0 = max(0, n - Wn)
+        want = np.stack([oracle.prefill_rows(Q[u], K[u], V[u], w.scale, [w.alpha], i0, n)[2][0]
+                         for u in range(U)])
+        got = to_f64(S1).reshape(U, n)
+        check_scores(got, want, rep, f"window {Wn}")
+        for u in range(U):
+            np.testing.assert_array_equal(kept1.cpu().numpy().reshape(U, -1)[u],
+                                          oracle.select(want[u], w.budget, w.recent))
+        bound = a2sf.a2sf_score_window_bound(w.alpha, n, Wn)
+        short = to_f64(S0).reshape(U, n) - got
+        assert short.min() >= -1e-4 * to_f64(S0).max() and short.max() <= bound * (1 + 1e-4) + 1e-30
+        if Wn >= n:
+            assert bound == 0.0 and torch.equal(S1, S0)
+
+
 # ---- the calls are asynchronous and hold no host-side state: a captured graph replays them ------
 @pytest.mark.parametrize("name,kw", [
     ("llama2_7b", dict(H=6, n=400, steps=12)),                                  # streaming kernel
@@ -307,6 +346,32 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     print(f"\n[streamed] {w.name}: units={U} n={n} M={w.budget} R={w.recent} evictions={evictions} "
           f"excused={excused} max_out={rep.max_out_err:.3g} max_score_rel={rep.max_score_rel:.3g}")
     cache.close()
+
+
+def test_several_tokens_in_one_call_equal_single_steps():
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W["llama2_7b"].scaled(H=4, n=300, budget=96, recent=40, steps=9)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    dq, dk, dv = wl.make_decode(w, device="cuda")                     # [T,B,H,d]
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    _, S, kept, _ = a2sf.a2sf_prefill(p, q, k, v)
+    one, many = a2sf.Cache(p), a2sf.Cache(p)
+    one.a2sf_cache_load(k, v, S, kept)
+    many.a2sf_cache_load(k, v, S, kept)
+    T = w.steps
+    o1 = torch.empty((T, w.B, w.H, w.d), dtype=q.dtype, device="cuda")
+    e1 = torch.empty((T, w.B, w.H), dtype=torch.int32, device="cuda")
+    for t in range(T):
+        one.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o1[t], e1[t])
+    tq, tk, tv = (x.permute(1, 2, 0, 3).contiguous() for x in (dq, dk, dv))      # [B,H,T,d]
+    o2, e2 = many.a2sf_decode_multi(w.alpha, tq, tk, tv)
+    torch.cuda.synchronize()
+    assert torch.equal(o2.permute(2, 0, 1, 3), o1) and torch.equal(e2, e1)
+    s1, s2 = one.a2sf_cache_export(), many.a2sf_cache_export()
+    torch.cuda.synchronize()
+    for key in ("scores", "pos", "count", "len", "k", "v"):
+        assert torch.equal(s1[key], s2[key]), key
 
 
 # ---- scoring pass that leaves out rows whose forgetting weight is exactly zero ------------------
