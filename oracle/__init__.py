@@ -228,3 +228,44 @@ def streaming_prefill(Q, K, V, scale: float, alpha, M: int, R: int, force=None, 
                                         force=None if force is None else force[i], nthreads=nthreads)
         out[:, i] = o
     return out, info, sc, cache
+
+
+def ideal_row(s_row: np.ndarray, keep: int) -> np.ndarray:
+    """Ideal pruning of one attention row (Sec. 4.3): of the row's logits the ``keep`` largest
+    stay (equal logits: the lower position first), the softmax runs over those alone.
+    Returns the full-length probability vector (zeros where pruned)."""
+    m = s_row.shape[0]
+    order = np.lexsort((np.arange(m), -s_row))[:min(keep, m)]
+    w = np.exp(s_row[order] - s_row[order].max())
+    p = np.zeros(m)
+    p[order] = w / w.sum()
+    return p
+
+
+def ideal_similarity(Q, K, V, scale: float, alpha, M: int, R: int, force=None, nthreads: int = 1,
+                     lib=None):
+    """Cosine similarity, row by row, between the attention a pruning policy actually uses while
+    the prompt streams through it and the ideal row that keeps the same number of tokens
+    (M cached + the token itself) by magnitude alone (Sec. 4.3, the similarity table).
+    Q, K, V: [U, n, d].  Returns (cos [U, n], out, info, scores, cache) with the last four as in
+    ``streaming_prefill``."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    U, n, d = Q.shape
+    cache = Cache(U, d, M, R, scale, lib=lib)
+    cos = np.empty((U, n), dtype=np.float64)
+    out = np.empty((U, n, d), dtype=np.float64)
+    info = np.empty((n, U, 3), dtype=np.int32)
+    sc = np.empty((n, U, 3), dtype=np.float64)
+    for i in range(n):
+        for u in range(U):
+            s_row = (K[u, :i + 1] @ Q[u, i]) * scale
+            seen = np.append(cache.pos[u, :cache.count[u]], i)          # cached tokens + itself
+            w = np.exp(s_row[seen] - s_row[seen].max())
+            meth = np.zeros(i + 1)
+            meth[seen] = w / w.sum()
+            ideal = ideal_row(s_row, M + 1)
+            cos[u, i] = (meth @ ideal) / np.sqrt((meth @ meth) * (ideal @ ideal))
+        o, info[i], sc[i] = cache.step(Q[:, i], K[:, i], V[:, i], alpha,
+                                        force=None if force is None else force[i], nthreads=nthreads)
+        out[:, i] = o
+    return cos, out, info, sc, cache

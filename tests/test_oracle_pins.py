@@ -482,3 +482,58 @@ def test_streamed_prompt_differs_from_one_shot_selection():
     dense = _brute_probs(Q, K, 0.35) @ V
     np.testing.assert_allclose(out[0, :9], dense[:9], rtol=1e-12, atol=1e-13)   # nothing evicted yet
     assert np.abs(out[0, 20:] - dense[20:]).max() > 1e-3
+
+
+# ---- similarity with the ideal mask (Sec. 4.3) --------------------------------------------------
+def test_ideal_row_is_a_top_k_softmax():
+    rng = np.random.default_rng(31)
+    s = rng.standard_normal(40)
+    s[7] = s[3]                                             # a tie: the lower position is kept first
+    for keep in (1, 5, 39, 40, 100):
+        p = oracle.ideal_row(s, keep)
+        k = min(keep, 40)
+        assert np.count_nonzero(p) == k and abs(p.sum() - 1) < 1e-14
+        kept = np.flatnonzero(p)
+        assert s[kept].min() >= np.delete(s, kept).max(initial=-np.inf)
+        t = torch.softmax(torch.from_numpy(s[kept]), 0).numpy()
+        np.testing.assert_allclose(p[kept], t, rtol=1e-13)
+    sel = np.zeros(40); sel[[3, 7]] = 1
+    s2 = np.where(sel > 0, 5.0, s - 10)                     # positions 3 and 7 tie at the top
+    assert np.flatnonzero(oracle.ideal_row(s2, 1)).tolist() == [3]
+
+
+def test_similarity_is_one_while_nothing_is_pruned_and_bounded_after():
+    rng = np.random.default_rng(32)
+    n, d, M = 30, 8, 10
+    Q, K, V = _rand_unit(rng, n, d)
+    cos, out, _, _, _ = oracle.ideal_similarity(Q[None], K[None], V[None], 0.35, 0.5, M=M, R=5)
+    np.testing.assert_allclose(cos[0, :M + 1], 1.0, rtol=0, atol=1e-14)   # rows that see every token
+    assert (cos > 0).all() and (cos <= 1 + 1e-14).all()
+    ref, _, _, _ = oracle.streaming_prefill(Q[None], K[None], V[None], 0.35, 0.5, M=M, R=5)
+    np.testing.assert_array_equal(out, ref)                                # the diagnostic changes nothing
+    full, *_ = oracle.ideal_similarity(Q[None], K[None], V[None], 0.35, 0.5, M=n, R=5)
+    np.testing.assert_allclose(full, 1.0, rtol=0, atol=1e-14)
+
+
+def test_similarity_orders_the_policies_on_a_sink_plus_recency_pattern():
+    """A prompt whose rows attend to token 0 (a sink), to two tokens that matter for a while and
+    to their neighbourhood: the sliding window loses the sink, pure accumulation (alpha = 1)
+    clings to early tokens, the forgetting factor follows the ideal mask most closely."""
+    rng = np.random.default_rng(33)
+    n, d, M = 96, 16, 12
+    K = rng.standard_normal((n, d))
+    Q = rng.standard_normal((n, d))
+    K[0] *= 0.2
+    e = np.zeros(d); e[0] = 6.0
+    K[0] += e; Q[:, 0] = 1.0                                   # every row likes token 0
+    for i in range(n):                                         # rows like a token some 20 rows back ...
+        j = max(0, i - 20 - (i % 7))
+        Q[i] += 0.9 * K[j]
+        if i >= 2:
+            Q[i] += 0.5 * K[i - 1]                             # ... and their predecessor
+    V = rng.standard_normal((n, d))
+    res = {}
+    for name, (alpha, R) in {"local": (1.0, M), "h2o": (1.0, M // 2), "a2sf": (0.6, 0)}.items():
+        cos, *_ = oracle.ideal_similarity(Q[None], K[None], V[None], 0.25, alpha, M=M, R=R)
+        res[name] = cos[0, M + 1:].mean()
+    assert res["local"] < res["h2o"] < res["a2sf"], res
