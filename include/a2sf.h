@@ -273,6 +273,28 @@ int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n,
                            int64_t stride_b, int64_t stride_h, int64_t stride_t,
                            void *out, int32_t *evicted_opt, void *cuda_stream);
 
+/* ---------------------------------------------------------------------------
+ * Similarity with the ideal mask (Sec. 4.3: the mask figure and the similarity table).
+ *
+ * Runs a2sf_prefill_streaming and, for every row i, compares the attention the policy
+ * actually uses -- the softmax over the cached tokens and token i itself -- with the ideal
+ * row: the softmax over the budget + 1 largest logits of ALL tokens 0..i (equal logits: the
+ * lower position first), i.e. the best any policy with that many tokens could do.
+ *     cos_out[b][h][i] = <a_i, p_i> / (|a_i| |p_i|),   both rows as length-(i+1) vectors.
+ * Rows i <= budget see every token and give 1.  Averaging (over rows, heads) is the caller's.
+ * q, k, v, out, evicted_opt as in a2sf_prefill_streaming; cos_out DEVICE [B][H][n] fp32.
+ * workspace: DEVICE, 256-byte aligned, a2sf_ideal_similarity_workspace_bytes (0 = invalid
+ * arguments).  n <= A2SF_IDEAL_SIMILARITY_MAX_N (a row's logits are held in shared memory).
+ * A diagnostic, not a hot path: 1 + 2n launches, O(n^2 d) CUDA-core work per unit.
+ * ------------------------------------------------------------------------- */
+#define A2SF_IDEAL_SIMILARITY_MAX_N 32768
+size_t a2sf_ideal_similarity_workspace_bytes(const a2sf_params *p, int32_t n);
+int a2sf_ideal_similarity(a2sf_cache *cache, float alpha, int32_t n,
+                          const void *q, const void *k, const void *v,
+                          int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                          void *out, float *cos_out, int32_t *evicted_opt,
+                          void *workspace, size_t workspace_bytes, void *cuda_stream);
+
 /* Snapshot / restore of the whole cache state into / from caller DEVICE buffers:
  * k, v [B][H][M][d] dtype; scores [B][H][M] fp32; pos [B][H][M] int32; count, len
  * [B][H] int32.  Any pointer may be NULL to skip that part. */

@@ -65,6 +65,8 @@ def _load():
         "a2sf_decode_step": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_decode_step_host": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_cache_reset": (ctypes.c_int, [vp, vp]),
+        "a2sf_ideal_similarity_workspace_bytes": (sz, [pp, i32]),
+        "a2sf_ideal_similarity": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]),
         "a2sf_score_window_bound": (ctypes.c_double, [f32, i32, i32]),
         "a2sf_decode_multi": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp]),
         "a2sf_prefill_streaming": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp]),
@@ -285,6 +287,25 @@ class Cache:
         (out [B,H,n,d], evicted [n,B,H] int32)."""
         return self._token_rows(lib.a2sf_prefill_streaming, "a2sf_prefill_streaming", alpha, q, k, v,
                                 out, evicted, stream)
+
+    def a2sf_ideal_similarity(self, alpha, q, k, v, stream=None):
+        """Streams the prompt through the policy and returns (cos [B,H,n] fp32, out, evicted):
+        per row, the cosine between the policy's attention and the ideal top-(budget+1) row."""
+        B, H, n, d = q.shape
+        assert (B, H, d) == (self.p.B, self.p.H, self.d) and q.dtype == self.torch_dtype
+        assert _strides(k) == _strides(q) and _strides(v) == _strides(q)
+        out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=q.device)
+        ev = torch.empty((n, B, H), dtype=torch.int32, device=q.device)
+        cos = torch.empty((B, H, n), dtype=torch.float32, device=q.device)
+        nbytes = int(lib.a2sf_ideal_similarity_workspace_bytes(ctypes.byref(self.p), n))
+        if nbytes == 0:
+            raise A2SFError(A2SF_ERR_INVALID_ARG, "a2sf_ideal_similarity_workspace_bytes")
+        ws = torch.empty((nbytes,), dtype=torch.uint8, device=q.device)
+        sb, sh, st = _strides(q)
+        _check(lib.a2sf_ideal_similarity(self.handle, alpha, n, _ptr(q), _ptr(k), _ptr(v), sb, sh, st,
+                                         _ptr(out), _ptr(cos), _ptr(ev), _ptr(ws), nbytes,
+                                         _stream(stream)), "a2sf_ideal_similarity")
+        return cos, out, ev
 
     def _token_rows(self, fn, name, alpha, q, k, v, out, evicted, stream):
         B, H, n, d = q.shape

@@ -420,6 +420,35 @@ int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n, const void
                              cuda_stream);
 }
 
+size_t a2sf_ideal_similarity_workspace_bytes(const a2sf_params *p, int32_t n)
+{
+    if (check_params(p) != A2SF_OK || n < 1 || n > A2SF_IDEAL_SIMILARITY_MAX_N) return 0;
+    return align_up(ideal_similarity_ws_bytes((size_t)p->B * p->H, n));
+}
+
+int a2sf_ideal_similarity(a2sf_cache *cache, float alpha, int32_t n, const void *q, const void *k,
+                          const void *v, int64_t stride_b, int64_t stride_h, int64_t stride_t,
+                          void *out, float *cos_out, int32_t *evicted_opt, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream)
+{
+    if (!cache || n < 1 || !q || !k || !v || !out || !cos_out) return A2SF_ERR_INVALID_ARG;
+    if (n > A2SF_IDEAL_SIMILARITY_MAX_N) return A2SF_ERR_UNSUPPORTED;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
+    int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
+    if (rc != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) || !aligned(cos_out, 4))
+        return A2SF_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256)) return A2SF_ERR_INVALID_ARG;
+    if (workspace_bytes < a2sf_ideal_similarity_workspace_bytes(&cache->p, n)) return A2SF_ERR_WORKSPACE;
+    rc = a2sf_cache_reset(cache, cuda_stream);
+    if (rc != A2SF_OK) return rc;
+    if (launch_ideal_similarity(cache->view, alpha, cache->p.H, n, q, k, v,
+                                Strides{stride_b, stride_h, stride_t}, out, cos_out, evicted_opt,
+                                cache->st_ev, workspace, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
 int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas, const void *q,
                               const void *k_new, const void *v_new, void *out,
                               int32_t *evicted_slot, void *cuda_stream)

@@ -163,4 +163,10 @@ __device__ __forceinline__ float unit_alpha(const float *alpha_vec, int u, float
 
 int read_and_clear_decode_status(cudaStream_t s);
 
+// similarity with the ideal mask while the prompt streams through the step kernel
+size_t ideal_similarity_ws_bytes(size_t units, int n);
+cudaError_t launch_ideal_similarity(const CacheView &view, float alpha, int H, int n, const void *q,
+                                    const void *k, const void *v, Strides st, void *out, float *cos_out,
+                                    int32_t *evicted, int32_t *ev_scratch, void *ws, cudaStream_t s);
+
 }  // namespace a2sf

@@ -348,6 +348,45 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     cache.close()
 
 
+# ---- similarity with the ideal mask ----------------------------------------------------------------
+@pytest.mark.parametrize("name,kw", [
+    ("tiny_fp32", dict()),                                                     # fp32, d = 64
+    ("llama2_7b", dict(H=4, n=300, budget=48, recent=24)),                     # bf16, half recent
+    ("opt_6p7b", dict(B=2, H=2, n=222, budget=40, recent=0, alpha=0.6)),       # fp16, the paper's split
+    ("llama2_7b", dict(H=3, n=150, budget=32, recent=32, alpha=1.0)),          # sliding window
+    ("llama2_13b", dict(B=1, H=2, n=90, budget=128, recent=64)),               # nothing pruned: all ones
+])
+def test_similarity_with_the_ideal_mask(name, kw):
+    import oracle
+    from parity_util import to_f64
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    cache, plain = a2sf.Cache(p), a2sf.Cache(p)
+    cos, out, ev = cache.a2sf_ideal_similarity(w.alpha, q, k, v)
+    out2, ev2 = plain.a2sf_prefill_streaming(w.alpha, q, k, v)
+    torch.cuda.synchronize()
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+    assert torch.equal(out, out2) and torch.equal(ev, ev2)           # the diagnostic changes nothing
+    U, n = w.units, w.n
+    ev_g = ev.cpu().numpy().reshape(n, U)
+    force = np.where(ev_g == -1, -3, ev_g).astype(np.int32)
+    Q, K, V = (to_f64(t).reshape(U, n, w.d) for t in (q, k, v))
+    want, *_ = oracle.ideal_similarity(Q, K, V, w.scale, w.alpha, w.budget, w.recent, force=force,
+                                       nthreads=oracle.host_threads())
+    got = cos.cpu().numpy().astype(np.float64).reshape(U, n)
+    # a pair of logits closer than fp32 resolves may swap at the ideal row's cut: the swapped
+    # probabilities are the row's smallest, so the cosine moves by far less than this
+    assert np.abs(got - want).max() <= 5e-4, np.abs(got - want).max()
+    assert abs(got.mean() - want.mean()) <= 2e-5
+    np.testing.assert_allclose(got[:, :min(n, w.budget + 1)], 1.0, rtol=0, atol=2e-6)
+    print(f"\n[similarity] {w.name} M={w.budget} R={w.recent} alpha={w.alpha}: mean cos over pruned rows "
+          f"{got[:, w.budget + 1:].mean() if n > w.budget + 1 else 1.0:.4f}, max |gpu-oracle| "
+          f"{np.abs(got - want).max():.2e}")
+
+
 def test_several_tokens_in_one_call_equal_single_steps():
     from paper_2407_20485_b200 import binding as a2sf
 
