@@ -269,3 +269,74 @@ def ideal_similarity(Q, K, V, scale: float, alpha, M: int, R: int, force=None, n
                                         force=None if force is None else force[i], nthreads=nthreads)
         out[:, i] = o
     return cos, out, info, sc, cache
+
+
+# ---- grouped query heads: G query heads share one K/V head and therefore one pruned cache ----------
+# The paper scores a token per head (Sec. 2.2); with a shared K/V head there is one set of tokens
+# to keep, and the reading taken here is that its score is the SUM of the group's attention
+# probabilities, accumulated and forgotten as in Eq. 5.
+
+def group_prefill(Q, K, V, scale: float, alpha: float, M: int, R: int, nthreads: int = 1, lib=None):
+    """Q [U, G, n, d] (U = batch x K/V heads), K, V [U, n, d].  Dense causal attention per query
+    head; S = sum over the group of each head's Eq. 5 scores; one selection per K/V head.
+    Returns out [U,G,n,d], lse [U,G,n], S [U,n], kept [U,min(n,M)]."""
+    Q, K, V = _f64(Q), _f64(K), _f64(V)
+    U, G, n, d = Q.shape
+    out = np.empty((U, G, n, d))
+    lse = np.empty((U, G, n))
+    S = np.zeros((U, n))
+    for g in range(G):
+        r = prefill(Q[:, g], K, V, scale, [alpha], M, R, nthreads=nthreads, lib=lib)
+        out[:, g], lse[:, g] = r["out"], r["lse"]
+        S += r["S"][:, 0]
+    kept = np.stack([select(S[u], M, R, lib=lib) for u in range(U)])
+    return {"out": out, "lse": lse, "S": S, "kept": kept}
+
+
+class GroupCache(Cache):
+    """The slot cache of ``Cache`` stepped by a group of query heads."""
+
+    def step_group(self, q, k_new, v_new, alpha: float, force=None):
+        """q [U, G, d]; k_new, v_new [U, d].  Steps (i)-(vi) of the generation step with G
+        softmaxes over the same cached tokens; a token's score gains the sum of the G
+        probabilities.  Returns out [U,G,d], info [U,3], scores [U,3] as ``Cache.step``."""
+        q, k_new, v_new = _f64(q), _f64(k_new), _f64(v_new)
+        U, G, d = q.shape
+        out = np.empty((U, G, d))
+        info = np.full((U, 3), -1, dtype=np.int32)
+        sc3 = np.zeros((U, 3))
+        for u in range(U):
+            cnt, p = int(self.count[u]), int(self.len[u])
+            Kall = np.vstack([self.K[u, :cnt], k_new[u:u + 1]])
+            Vall = np.vstack([self.V[u, :cnt], v_new[u:u + 1]])
+            gain = np.zeros(cnt + 1)
+            for g in range(G):
+                t = (Kall @ q[u, g]) * self.scale
+                a = np.exp(t - t.max())
+                a /= a.sum()
+                out[u, g] = a @ Vall
+                gain += a
+            self.S[u, :cnt] = alpha * self.S[u, :cnt] + gain[:cnt]
+            s_new = gain[cnt]
+            if cnt < self.M:
+                target = cnt
+                self.count[u] = cnt + 1
+            else:
+                cand = [(self.S[u, s], int(self.pos[u, s]), s) for s in range(cnt)
+                        if self.pos[u, s] <= p - self.R]
+                if self.R == 0:
+                    cand.append((s_new, p, -2))
+                cand.sort(key=lambda c: (c[0], c[1]))
+                info[u, 1], sc3[u, 1] = cand[0][2], cand[0][0]
+                if len(cand) > 1:
+                    info[u, 2], sc3[u, 2] = cand[1][2], cand[1][0]
+                target = cand[0][2]
+                if force is not None and force[u] != -3:
+                    target = int(force[u])
+                info[u, 0] = target
+                sc3[u, 0] = s_new if target == -2 else self.S[u, target]
+            if target >= 0:
+                self.K[u, target], self.V[u, target] = k_new[u], v_new[u]
+                self.S[u, target], self.pos[u, target] = s_new, p
+            self.len[u] = p + 1
+        return out, info, sc3

@@ -113,6 +113,7 @@ static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.lse = lse_opt ? lse_opt : static_cast<float *>(workspace);
     a.scores = scores;
     a.st = Strides{stride_b, stride_h, stride_t};
+    a.st_kv = a.st; a.G = 1;
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
@@ -164,6 +165,7 @@ static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const vo
     a.lse = const_cast<float *>(lse);
     a.scores = scores;
     a.st = Strides{stride_b, stride_h, stride_t};
+    a.st_kv = a.st; a.G = 1;
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = alpha_vec;
     a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;

@@ -102,8 +102,10 @@ struct PrefillArgs {
     void *out;
     float *lse;        // [U][n]
     float *scores;     // [U][n]
-    Strides st;
-    int B, H, n, d;
+    Strides st;        // of q and out
+    Strides st_kv;     // of k and v ([B][H/G][n][d]); equal to st without head grouping
+    int B, H, n, d;    // H = query heads
+    int G;             // query heads per key/value head (1 = one K/V head per query head)
     float scale, alpha;
     const float *alpha_vec;   // per-unit forgetting factors [U] on the device, or nullptr (use alpha)
     int skip_zero_rows;       // scoring pass: leave out rows whose weight is exactly 0 in fp32

@@ -80,9 +80,10 @@ __global__ void __launch_bounds__(kThreads) prefill_pass1_simt(PrefillArgs a)
     const int u = blockIdx.x;
     const int b = u / a.H, h = u % a.H;
     const int64_t base = (int64_t)b * a.st.b + (int64_t)h * a.st.h;
+    const int64_t base_kv = (int64_t)b * a.st_kv.b + (int64_t)(h / a.G) * a.st_kv.h;   // shared K/V head
     const T *Q = static_cast<const T *>(a.q) + base;
-    const T *K = static_cast<const T *>(a.k) + base;
-    const T *V = static_cast<const T *>(a.v) + base;
+    const T *K = static_cast<const T *>(a.k) + base_kv;
+    const T *V = static_cast<const T *>(a.v) + base_kv;
     T *O = static_cast<T *>(a.out) + base;
 
     const int tq = threadIdx.x & 3;
@@ -98,8 +99,8 @@ __global__ void __launch_bounds__(kThreads) prefill_pass1_simt(PrefillArgs a)
     const int last_row = min(a.n, (rb + 1) * kRows) - 1;
     for (int j0 = 0; j0 <= last_row; j0 += kTile) {
         __syncthreads();
-        load_tile<T, D>(Ks, K, a.st.t, j0, a.n);
-        load_tile<T, D>(Vs, V, a.st.t, j0, a.n);
+        load_tile<T, D>(Ks, K, a.st_kv.t, j0, a.n);
+        load_tile<T, D>(Vs, V, a.st_kv.t, j0, a.n);
         __syncthreads();
         float s[kTile];
         float tmax = -INFINITY;
@@ -153,8 +154,9 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
     const int u = blockIdx.x;
     const int b = u / a.H, h = u % a.H;
     const int64_t base = (int64_t)b * a.st.b + (int64_t)h * a.st.h;
+    const int64_t base_kv = (int64_t)b * a.st_kv.b + (int64_t)(h / a.G) * a.st_kv.h;
     const T *Q = static_cast<const T *>(a.q) + base;
-    const T *K = static_cast<const T *>(a.k) + base;
+    const T *K = static_cast<const T *>(a.k) + base_kv;
     const float *lse = a.lse + (int64_t)u * a.n;
 
     const int tq = threadIdx.x & 3;
@@ -162,7 +164,7 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
     const bool valid = j < a.n;
 
     float kv[D / 4];
-    load_own_row<T, D>(kv, K + (int64_t)j * a.st.t, tq, valid);
+    load_own_row<T, D>(kv, K + (int64_t)j * a.st_kv.t, tq, valid);
 
     // weight alpha^(n-1-i) folded into the exponent: exp2(s*log2e - c_i),
     // c_i = lse_i*log2e - (n-1-i)*log2(alpha); alpha = 0 keeps only row n-1 (0^0 = 1).

@@ -79,6 +79,7 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
     a.lse = lse;          // every row this call reads is written by its own first pass,
     a.scores = scores;    // so nothing has to be cleared between calls
     a.st = Strides{stride_b, stride_h, stride_t};
+    a.st_kv = a.st; a.G = 1;
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
     a.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
     a.alpha = p->alpha;

@@ -42,6 +42,7 @@ struct ScoreArgs {
     const float *lse;     // [U][n]
     float *scores;        // [U][n]
     int n, H;
+    int G;                // query heads per key/value head
     float sl2;            // scale * log2(e)
     float alpha;          // forgetting factor, or per unit:
     const float *alpha_vec;
@@ -187,8 +188,8 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             prefetch_tmap(&tmap_q);
             prefetch_tmap(&tmap_k);
             mbar_arrive_expect_tx(&sh->k_full, kTileBytes);
-            tma_load_4d(Ks, &tmap_k, &sh->k_full, 0, kb * kBlk, h, b);
-            tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full, 64, kb * kBlk, h, b);
+            tma_load_4d(Ks, &tmap_k, &sh->k_full, 0, kb * kBlk, h / a.G, b);
+            tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full, 64, kb * kBlk, h / a.G, b);
         }
         int issued = 0;
         for (int it = 0; it < ntiles; ++it) {
@@ -339,6 +340,7 @@ struct AttnArgs {
     float *lse;           // [U][n]
     int64_t st_b, st_h, st_t;
     int n, H;
+    int G;                // query heads per key/value head
     float sl2;            // scale * log2(e)
     const int *v_flag;    // bf16 storage: 0 = the fp16 copy of V is exact, 1 = it is not
     int run_if_flag;      // this launch works only when *v_flag equals this value
@@ -462,18 +464,19 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 tma_load_4d(Qs + kTileBytes, &tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
                 tma_load_4d(Qs + kTileBytes + kHalfBytes, &tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
             }
+            const int hk = h / a.G;                   // the K/V head this query head reads
             int k_issued = 0, v_issued = 0;
             for (int t = 0; t < nt; ++t) {
                 const int ks = t % kKStages, vs = t % kVStages;
                 if (!wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
-                tma_load_4d(Ks + ks * kTileBytes, &tmap_k, &sh->k_full[ks], 0, t * kBlk, h, b);
-                tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[ks], 64, t * kBlk, h, b);
+                tma_load_4d(Ks + ks * kTileBytes, &tmap_k, &sh->k_full[ks], 0, t * kBlk, hk, b);
+                tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[ks], 64, t * kBlk, hk, b);
                 k_issued = t + 1;
                 if (!wait(&sh->v_empty[vs], ((t / kVStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->v_full[vs], kTileBytes);
-                tma_load_4d(Vs + vs * kTileBytes, &tmap_v, &sh->v_full[vs], 0, t * kBlk, h, b);
-                tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[vs], 64, t * kBlk, h, b);
+                tma_load_4d(Vs + vs * kTileBytes, &tmap_v, &sh->v_full[vs], 0, t * kBlk, hk, b);
+                tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[vs], 64, t * kBlk, hk, b);
                 v_issued = t + 1;
             }
             if (*abort_flag) {
@@ -746,13 +749,12 @@ EncodeTiledFn encode_fn()
 
 // [B][H][n][d] 16-bit tensor -> 4-D map (d, n, H, B), box 64 x 128 rows, 128-byte swizzle,
 // out-of-range rows read as zero.
-bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillArgs &a,
-                   const Strides *override_strides = nullptr)
+bool make_tile_map(CUtensorMap *map, int dtype, const void *base, const PrefillArgs &a, int heads,
+                   const Strides &st)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
-    const Strides st = override_strides ? *override_strides : a.st;
-    const cuuint64_t dims[4] = {(cuuint64_t)a.d, (cuuint64_t)a.n, (cuuint64_t)a.H, (cuuint64_t)a.B};
+    const cuuint64_t dims[4] = {(cuuint64_t)a.d, (cuuint64_t)a.n, (cuuint64_t)heads, (cuuint64_t)a.B};
     const cuuint64_t strides[3] = {(cuuint64_t)st.t * 2, (cuuint64_t)st.h * 2, (cuuint64_t)st.b * 2};
     const cuuint32_t box[4] = {64, (cuuint32_t)kBlk, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -780,8 +782,9 @@ size_t prefill_tc_extra_bytes(int dtype, size_t units, int n, int d)
 cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
 {
     CUtensorMap mq, mk, mv;
-    if (!make_tile_map(&mq, dtype, a.q, a) || !make_tile_map(&mk, dtype, a.k, a) ||
-        !make_tile_map(&mv, dtype, a.v, a))
+    const int Hkv = a.H / a.G;
+    if (!make_tile_map(&mq, dtype, a.q, a, a.H, a.st) || !make_tile_map(&mk, dtype, a.k, a, Hkv, a.st_kv) ||
+        !make_tile_map(&mv, dtype, a.v, a, Hkv, a.st_kv))
         return cudaErrorInvalidValue;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -797,7 +800,7 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     AttnArgs aa;
     aa.out = a.out; aa.lse = a.lse;
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
-    aa.n = a.n; aa.H = a.H;
+    aa.n = a.n; aa.H = a.H; aa.G = a.G;
     aa.sl2 = a.scale * kLog2e;
     aa.v_flag = nullptr; aa.run_if_flag = 0;
     const int npairs = ((a.n + kBlk - 1) / kBlk + 1) / 2;
@@ -816,15 +819,15 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     // the copy decides on the device which of the two does the work (no host round trip)
     cudaError_t e = cudaMemsetAsync(a.v_flag, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
-    const size_t chunks = (size_t)a.B * a.H * a.n * (kD / 8);
+    const size_t chunks = (size_t)a.B * Hkv * a.n * (kD / 8);
     const unsigned cgrid = (unsigned)std::min<size_t>((chunks + 255) / 256, 148 * 16);
-    v_to_half_kernel<<<cgrid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(a.v), a.st, a.H, a.n, chunks,
+    v_to_half_kernel<<<cgrid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(a.v), a.st_kv, Hkv, a.n, chunks,
                                            static_cast<__half *>(a.v_half), a.v_flag);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    const Strides contig{(int64_t)a.H * a.n * kD, (int64_t)a.n * kD, (int64_t)kD};
+    const Strides contig{(int64_t)Hkv * a.n * kD, (int64_t)a.n * kD, (int64_t)kD};
     CUtensorMap mvh;
-    if (!make_tile_map(&mvh, A2SF_F16, a.v_half, a, &contig)) return cudaErrorInvalidValue;
+    if (!make_tile_map(&mvh, A2SF_F16, a.v_half, a, Hkv, contig)) return cudaErrorInvalidValue;
     aa.v_flag = a.v_flag;
     aa.run_if_flag = 0;
     attn_pass_tc<__nv_bfloat16, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mvh, aa);
@@ -839,7 +842,8 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s)
 {
     CUtensorMap mq, mk;
-    if (!make_tile_map(&mq, dtype, a.q, a) || !make_tile_map(&mk, dtype, a.k, a))
+    if (!make_tile_map(&mq, dtype, a.q, a, a.H, a.st) ||
+        !make_tile_map(&mk, dtype, a.k, a, a.H / a.G, a.st_kv))
         return cudaErrorInvalidValue;
     static std::once_flag once;
     static cudaError_t attr_err = cudaSuccess;
@@ -849,7 +853,7 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     });
     if (attr_err != cudaSuccess) return attr_err;
     ScoreArgs sa;
-    sa.lse = a.lse; sa.scores = a.scores; sa.n = a.n; sa.H = a.H;
+    sa.lse = a.lse; sa.scores = a.scores; sa.n = a.n; sa.H = a.H; sa.G = a.G;
     sa.sl2 = a.scale * kLog2e;
     sa.alpha = a.alpha;
     sa.alpha_vec = a.alpha_vec;

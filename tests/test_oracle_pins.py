@@ -537,3 +537,64 @@ def test_similarity_orders_the_policies_on_a_sink_plus_recency_pattern():
         cos, *_ = oracle.ideal_similarity(Q[None], K[None], V[None], 0.25, alpha, M=M, R=R)
         res[name] = cos[0, M + 1:].mean()
     assert res["local"] < res["h2o"] < res["a2sf"], res
+
+
+# ---- grouped query heads ------------------------------------------------------------------------
+def test_group_of_one_is_the_single_head_step():
+    rng = np.random.default_rng(41)
+    U, d, M, R = 3, 8, 6, 2
+    K, V = rng.standard_normal((2, U, M, d))
+    S = rng.random((U, M))
+    kept = np.tile(np.arange(M, dtype=np.int32), (U, 1))
+    a, b = oracle.Cache(U, d, M, R, 0.3), oracle.GroupCache(U, d, M, R, 0.3)
+    a.load(K, V, S, kept); b.load(K, V, S, kept)
+    for t in range(8):
+        q, k, v = rng.standard_normal((3, U, d))
+        o1, i1, s1 = a.step(q, k, v, 0.6)
+        o2, i2, s2 = b.step_group(q[:, None], k, v, 0.6)
+        np.testing.assert_allclose(o2[:, 0], o1, rtol=1e-13, atol=1e-15)
+        np.testing.assert_array_equal(i2, i1)
+        np.testing.assert_allclose(s2, s1, rtol=1e-13)
+        np.testing.assert_allclose(b.S, a.S, rtol=1e-13)
+        np.testing.assert_array_equal(b.pos, a.pos)
+
+
+def test_group_scores_are_the_sum_of_the_heads_attention():
+    """Prefill: S = sum_g of Eq. 5 per head, from independently built attention matrices.
+    Decode without eviction: prefill(n) + T grouped steps == prefill(n + T)."""
+    rng = np.random.default_rng(42)
+    G, n, T, d, alpha, scale = 3, 14, 6, 8, 0.7, 0.3
+    Q = rng.standard_normal((G, n + T, d))
+    K, V = rng.standard_normal((2, n + T, d))
+    K[0] *= 3
+    full = oracle.group_prefill(Q[None], K[None], V[None], scale, alpha, M=64, R=4)
+    want = sum(_brute_scores(_brute_probs(Q[g], K, scale), alpha) for g in range(G))
+    np.testing.assert_allclose(full["S"][0], want, rtol=1e-12)
+    for g in range(G):
+        np.testing.assert_allclose(full["out"][0, g], _brute_probs(Q[g], K, scale) @ V, rtol=1e-12, atol=1e-14)
+    head = oracle.group_prefill(Q[None, :, :n], K[None, :n], V[None, :n], scale, alpha, M=64, R=4)
+    c = oracle.GroupCache(1, d, 64, 4, scale)
+    c.load(K[None, :n], V[None, :n], head["S"], head["kept"])
+    for t in range(n, n + T):
+        o, info, _ = c.step_group(Q[None, :, t], K[None, t], V[None, t], alpha)
+        np.testing.assert_allclose(o[0], full["out"][0, :, t], rtol=1e-12, atol=1e-14)
+        assert info[0, 0] == -1
+    np.testing.assert_allclose(c.S[0, :n + T], full["S"][0], rtol=1e-12)
+
+
+def test_group_eviction_follows_the_summed_score():
+    """Two heads that each favour a different old token keep both; the token neither looks at goes."""
+    d, M = 4, 3
+    e = np.eye(d)
+    K = np.stack([e[0], e[1], e[2]]) * 4.0
+    c = oracle.GroupCache(1, d, M, 1, 1.0)
+    c.load(K[None], K[None], np.full((1, 3), 0.5), np.arange(3, dtype=np.int32)[None])
+    q = np.stack([e[0], e[1]]) * 4.0                       # head 0 -> token 0, head 1 -> token 1
+    out, info, sc = c.step_group(q[None], (e[3] * 4.0)[None], e[3][None], 0.5)
+    assert info[0, 0] == 2                                  # token 2 had the lowest summed score
+    assert sorted(c.pos[0].tolist()) == [0, 1, 3]
+    # the same step with a single head (head 0 only) would have dropped token 1 or 2, lowest position first
+    c1 = oracle.GroupCache(1, d, M, 1, 1.0)
+    c1.load(K[None], K[None], np.full((1, 3), 0.5), np.arange(3, dtype=np.int32)[None])
+    _, info1, _ = c1.step_group(q[None, :1], (e[3] * 4.0)[None], e[3][None], 0.5)
+    assert info1[0, 0] == 1
