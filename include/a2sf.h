@@ -251,6 +251,37 @@ int a2sf_decode_multi(a2sf_cache *cache, float alpha, int32_t steps,
                       int64_t stride_b, int64_t stride_h, int64_t stride_t,
                       void *out, int32_t *evicted_opt, void *cuda_stream);
 
+/* ---------------------------------------------------------------------------
+ * Grouped query heads (GQA / MQA): `group` query heads share one K/V head, hence one pruned
+ * cache.  The paper scores tokens per head and leaves grouping open (Limitation section);
+ * the rule here: a token's score is the SUM over the group's query heads of Eq. 5, and one
+ * selection / one eviction per K/V head serves the whole group.  a2sf_params.H counts K/V
+ * heads; the query tensors have H * group heads, head h*group + g reading K/V head h.
+ *
+ * a2sf_prefill_group: q, out DEVICE [B][H*group][n][d] (q strides), k, v DEVICE [B][H][n][d]
+ * (kv strides), scores [B][H][n] fp32 (summed over the group), kept_idx [B][H][min(n,budget)],
+ * lse_opt [B][H*group][n] or NULL.  flags and score_window must be 0.  Workspace as for
+ * a2sf_prefill, size from a2sf_prefill_group_workspace_bytes (0 = invalid arguments).
+ *
+ * a2sf_decode_step_group: the generation step for a cache built from those scores
+ * (a2sf_cache_load).  q, out DEVICE [B][H*group][d] contiguous; k_new, v_new DEVICE [B][H][d];
+ * evicted_slot [B][H].  Each query head attends over the cached tokens and the new one; the
+ * cached scores become alpha * S + sum_g a_g, the new token's score sum_g a_g,self; eviction as
+ * in a2sf_decode_step.  A2SF_ERR_UNSUPPORTED when group > A2SF_MAX_GROUP or group * budget is
+ * too large for one CTA's shared memory (about 50,000 slots x heads).
+ * ------------------------------------------------------------------------- */
+#define A2SF_MAX_GROUP 8
+size_t a2sf_prefill_group_workspace_bytes(const a2sf_params *p, int32_t group, int32_t n);
+int a2sf_prefill_group(const a2sf_params *p, int32_t group, int32_t n,
+                       const void *q, int64_t q_stride_b, int64_t q_stride_h, int64_t q_stride_t,
+                       const void *k, const void *v,
+                       int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t,
+                       void *out, float *scores, int32_t *kept_idx, float *lse_opt,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+int a2sf_decode_step_group(a2sf_cache *cache, int32_t group, float alpha,
+                           const void *q, const void *k_new, const void *v_new,
+                           void *out, int32_t *evicted_slot, void *cuda_stream);
+
 /* Empties the cache (count = length = 0, scores 0, positions -1), asynchronously. */
 int a2sf_cache_reset(a2sf_cache *cache, void *cuda_stream);
 

@@ -65,6 +65,10 @@ def _load():
         "a2sf_decode_step": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_decode_step_host": (ctypes.c_int, [vp, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_cache_reset": (ctypes.c_int, [vp, vp]),
+        "a2sf_prefill_group_workspace_bytes": (sz, [pp, i32, i32]),
+        "a2sf_prefill_group": (ctypes.c_int, [pp, i32, i32, vp, i64, i64, i64, vp, vp, i64, i64, i64,
+                                              vp, vp, vp, vp, vp, sz, vp]),
+        "a2sf_decode_step_group": (ctypes.c_int, [vp, i32, f32, vp, vp, vp, vp, vp, vp]),
         "a2sf_ideal_similarity_workspace_bytes": (sz, [pp, i32]),
         "a2sf_ideal_similarity": (ctypes.c_int, [vp, f32, i32, vp, vp, vp, i64, i64, i64, vp, vp, vp, vp, sz, vp]),
         "a2sf_score_window_bound": (ctypes.c_double, [f32, i32, i32]),
@@ -173,6 +177,27 @@ def a2sf_prefill(p: a2sf_params, q, k, v, out=None, scores=None, kept_idx=None, 
     return out, scores, kept_idx, lse
 
 
+def a2sf_prefill_group(p: a2sf_params, group: int, q, k, v, stream=None):
+    """Grouped query heads: q [B, H*group, n, d], k, v [B, H, n, d] (p.H = K/V heads).
+    Returns (out [B,H*group,n,d], scores [B,H,n], kept_idx [B,H,m], lse [B,H*group,n])."""
+    B, Hq, n, d = q.shape
+    assert Hq == p.H * group and k.shape == (B, p.H, n, d) and v.shape == k.shape
+    assert _strides(v) == _strides(k)
+    dev = q.device
+    out = torch.empty_strided(q.shape, q.stride(), dtype=q.dtype, device=dev)
+    scores = torch.empty((B, p.H, n), dtype=torch.float32, device=dev)
+    kept = torch.empty((B, p.H, min(n, p.budget)), dtype=torch.int32, device=dev)
+    lse = torch.empty((B, Hq, n), dtype=torch.float32, device=dev)
+    nbytes = int(lib.a2sf_prefill_group_workspace_bytes(ctypes.byref(p), group, n))
+    if nbytes == 0:
+        raise A2SFError(A2SF_ERR_INVALID_ARG, "a2sf_prefill_group_workspace_bytes")
+    ws = torch.empty((nbytes,), dtype=torch.uint8, device=dev)
+    _check(lib.a2sf_prefill_group(ctypes.byref(p), group, n, _ptr(q), *_strides(q), _ptr(k), _ptr(v),
+                                  *_strides(k), _ptr(out), _ptr(scores), _ptr(kept), _ptr(lse), _ptr(ws),
+                                  nbytes, _stream(stream)), "a2sf_prefill_group")
+    return out, scores, kept, lse
+
+
 def a2sf_rescore(p: a2sf_params, q, k, lse, scores=None, kept_idx=None, workspace=None,
                  stream=None, alphas=None):
     """Scores and kept set for ``p.alpha`` from an existing log-sum-exp."""
@@ -268,6 +293,13 @@ class Cache:
         _check(lib.a2sf_decode_step_per_head(self.handle, _ptr(alphas), _ptr(q), _ptr(k_new), _ptr(v_new),
                                              _ptr(out), _ptr(evicted), _stream(stream)),
                "a2sf_decode_step_per_head")
+
+    def a2sf_decode_step_group(self, group, alpha, q, k_new, v_new, out, evicted, stream=None):
+        """q, out [B, H*group, d]; k_new, v_new [B, H, d]; evicted [B, H]."""
+        assert q.is_contiguous() and out.is_contiguous() and k_new.is_contiguous() and v_new.is_contiguous()
+        _check(lib.a2sf_decode_step_group(self.handle, group, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),
+                                          _ptr(out), _ptr(evicted), _stream(stream)),
+               "a2sf_decode_step_group")
 
     def a2sf_decode_step_host(self, alpha, q, k_new, v_new, out, evicted, stream=None):
         _check(lib.a2sf_decode_step_host(self.handle, alpha, _ptr(q), _ptr(k_new), _ptr(v_new),

@@ -139,6 +139,69 @@ int a2sf_prefill(const a2sf_params *p, int32_t n, const void *q, const void *k, 
                         lse_opt, workspace, workspace_bytes, cuda_stream);
 }
 
+// workspace of the grouped prefill: lse rows and per-query-head scores [B][H*G][n], then the
+// tensor-core pass's own extra (the fp16 copy of the B*H K/V heads' V)
+static size_t group_ws_bytes(const a2sf_params *p, int G, int n)
+{
+    const size_t rows = align_up((size_t)p->B * p->H * G * n * sizeof(float));
+    return 2 * rows + prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d);
+}
+
+size_t a2sf_prefill_group_workspace_bytes(const a2sf_params *p, int32_t group, int32_t n)
+{
+    if (check_params(p) != A2SF_OK || n < 1 || group < 1 || group > A2SF_MAX_GROUP) return 0;
+    return group_ws_bytes(p, group, n);
+}
+
+int a2sf_prefill_group(const a2sf_params *p, int32_t group, int32_t n, const void *q, int64_t q_stride_b,
+                       int64_t q_stride_h, int64_t q_stride_t, const void *k, const void *v,
+                       int64_t kv_stride_b, int64_t kv_stride_h, int64_t kv_stride_t, void *out,
+                       float *scores, int32_t *kept_idx, float *lse_opt, void *workspace,
+                       size_t workspace_bytes, void *cuda_stream)
+{
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (group < 1 || group > A2SF_MAX_GROUP) return A2SF_ERR_UNSUPPORTED;
+    if (p->score_window != 0 || p->flags != 0) return A2SF_ERR_UNSUPPORTED;
+    if (n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    if ((rc = check_strides(p, q_stride_b, q_stride_h, q_stride_t)) != A2SF_OK) return rc;
+    if ((rc = check_strides(p, kv_stride_b, kv_stride_h, kv_stride_t)) != A2SF_OK) return rc;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) ||
+        !aligned(scores, 4) || !aligned(kept_idx, 4))
+        return A2SF_ERR_INVALID_ARG;
+    if (!workspace || !aligned(workspace, 256)) return A2SF_ERR_INVALID_ARG;
+    if (workspace_bytes < group_ws_bytes(p, group, n)) return A2SF_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const size_t rows = align_up((size_t)p->B * p->H * group * n * sizeof(float));
+    char *ws = static_cast<char *>(workspace);
+
+    PrefillArgs a;
+    a.q = q; a.k = k; a.v = v; a.out = out;
+    a.lse = lse_opt ? lse_opt : reinterpret_cast<float *>(ws);
+    a.scores = reinterpret_cast<float *>(ws + rows);              // one row per QUERY head
+    a.st = Strides{q_stride_b, q_stride_h, q_stride_t};
+    a.st_kv = Strides{kv_stride_b, kv_stride_h, kv_stride_t};
+    a.G = group;
+    a.B = p->B; a.H = p->H * group; a.n = n; a.d = p->d;
+    a.scale = eff_scale(p); a.alpha = p->alpha; a.alpha_vec = nullptr;
+    a.skip_zero_rows = 0; a.window_rows = 0;
+    a.v_half = nullptr; a.v_flag = nullptr;
+    if (prefill_tc_extra_bytes(p->dtype, (size_t)p->B * p->H, n, p->d) > 0) {
+        a.v_flag = reinterpret_cast<int *>(ws + 2 * rows);
+        a.v_half = ws + 2 * rows + 256;
+    }
+    const bool tc = prefill_tc_supported(p->dtype, a);
+    if ((tc ? launch_prefill_pass1_tc(p->dtype, a, s) : launch_prefill_pass1_simt(p->dtype, a, s)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if ((tc ? launch_prefill_pass2_tc(p->dtype, a, s) : launch_prefill_pass2_simt(p->dtype, a, s)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if (launch_group_sum(a.scores, scores, group, n, (size_t)p->B * p->H, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if (launch_select(scores, kept_idx, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
 int a2sf_prefill_per_head(const a2sf_params *p, int32_t n, const void *q, const void *k, const void *v,
                           int64_t stride_b, int64_t stride_h, int64_t stride_t, const float *alphas,
                           void *out, float *scores, int32_t *kept_idx, float *lse_opt,
@@ -447,6 +510,21 @@ int a2sf_ideal_similarity(a2sf_cache *cache, float alpha, int32_t n, const void 
     if (launch_ideal_similarity(cache->view, alpha, cache->p.H, n, q, k, v,
                                 Strides{stride_b, stride_h, stride_t}, out, cos_out, evicted_opt,
                                 cache->st_ev, workspace, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_decode_step_group(a2sf_cache *cache, int32_t group, float alpha, const void *q, const void *k_new,
+                           const void *v_new, void *out, int32_t *evicted_slot, void *cuda_stream)
+{
+    if (!cache || !q || !k_new || !v_new || !out || !evicted_slot) return A2SF_ERR_INVALID_ARG;
+    if (group < 1 || group > A2SF_MAX_GROUP) return A2SF_ERR_UNSUPPORTED;
+    if (decode_group_smem_bytes(cache->view.M, group, cache->view.d) > 220 * 1024) return A2SF_ERR_UNSUPPORTED;
+    if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16))
+        return A2SF_ERR_INVALID_ARG;
+    if (launch_decode_step_group(cache->view, group, alpha, q, k_new, v_new, out, evicted_slot,
+                                 static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return A2SF_ERR_CUDA;
     return A2SF_OK;
 }

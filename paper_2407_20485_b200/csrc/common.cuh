@@ -165,6 +165,12 @@ __device__ __forceinline__ float unit_alpha(const float *alpha_vec, int u, float
 
 int read_and_clear_decode_status(cudaStream_t s);
 
+// grouped query heads (G query heads per K/V head)
+cudaError_t launch_group_sum(const float *per_head, float *out, int G, int n, size_t units, cudaStream_t s);
+size_t decode_group_smem_bytes(int M, int G, int d);
+cudaError_t launch_decode_step_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                                     const void *v_new, void *out, int32_t *evicted, cudaStream_t s);
+
 // similarity with the ideal mask while the prompt streams through the step kernel
 size_t ideal_similarity_ws_bytes(size_t units, int n);
 cudaError_t launch_ideal_similarity(const CacheView &view, float alpha, int H, int n, const void *q,

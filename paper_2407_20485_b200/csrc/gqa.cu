@@ -1,0 +1,283 @@
+// Grouped query heads: G query heads share one K/V head and therefore one pruned cache.
+// The paper scores tokens per head (Sec. 2.2) and leaves head grouping open (Limitation
+// section); here a cached token's score gains, per step, the SUM of the group's attention
+// probabilities, and one eviction serves the whole group.
+//
+//   group_sum_kernel       : prefill scores of the G query heads -> one score row per K/V head.
+//   decode_step_group_kernel: the generation step for one K/V unit and its G queries.  K and V
+//                            rows are read once; each lane keeps its 16-byte slice of all G
+//                            queries in registers, so the extra heads cost arithmetic, not
+//                            memory traffic.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace a2sf {
+namespace {
+
+constexpr int kGroupThreads = 256;
+constexpr int kMaxGroup = 8;
+
+__global__ void group_sum_kernel(const float *__restrict__ per_head, float *__restrict__ out, int G, int n,
+                                 size_t total)
+{
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (size_t)gridDim.x * blockDim.x) {
+        const size_t u = idx / n, j = idx % n;
+        float s = 0.f;
+        for (int g = 0; g < G; ++g) s += per_head[(u * G + g) * (size_t)n + j];   // fixed order
+        out[idx] = s;
+    }
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kGroupThreads)
+decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ q,
+                         const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ out,
+                         int32_t *__restrict__ evicted)
+{
+    constexpr int VEC = Elem<T>::kVec;
+    constexpr int LPR = D / VEC;              // lanes per row
+    constexpr int RPW = 32 / LPR;             // rows per warp-wide load
+    constexpr int NW = kGroupThreads / 32;
+    const int M = c.M;
+    const int wstride = (M + 1 + 3) & ~3;     // floats per query head in w[]
+
+    extern __shared__ __align__(16) float gsm[];
+    float *w = gsm;                                   // [G][wstride] logits, then probabilities
+    float *part = w + (size_t)G * wstride;            // [NW][G][D] partial outputs
+    __shared__ unsigned long long red_key[NW];
+    __shared__ int red_slot[NW];
+    __shared__ int s_target;
+
+    const int u = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int sub = lane % LPR, rsel = lane / LPR;
+    const int cnt = min(c.count[u], M);
+    const int p = c.len[u];
+    T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
+    T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
+    float *Su = c.S + (size_t)u * M;
+    int32_t *posu = c.pos + (size_t)u * M;
+    const T *qu = q + (size_t)u * G * D;              // [G][D]
+    const T *knu = k_new + (size_t)u * D, *vnu = v_new + (size_t)u * D;
+
+    // this lane's slice of every query
+    float qf[kMaxGroup][VEC];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g)
+        if (g < G) Elem<T>::unpack(*reinterpret_cast<const uint4 *>(qu + (size_t)g * D + sub * VEC), qf[g]);
+
+    // ---- (i) logits of the cached keys and of the new key, for every query of the group -----
+    // kUnroll row groups per iteration, their loads issued before any arithmetic
+    constexpr int kUnroll = 4;
+    for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
+        uint4 raw[kUnroll];
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int s = s0 + x * NW * RPW + rsel;
+            raw[x] = make_uint4(0u, 0u, 0u, 0u);
+            if (s <= cnt)
+                raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? Ku + (size_t)s * D : knu) + sub * VEC);
+        }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int s = s0 + x * NW * RPW + rsel;
+            float kf[VEC];
+            Elem<T>::unpack(raw[x], kf);
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                if (g < G) {
+                    float dot = 0.f;
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) dot = fmaf(qf[g][e], kf[e], dot);
+#pragma unroll
+                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                    if (sub == 0 && s <= cnt) w[g * wstride + s] = dot * c.scale;
+                }
+            }
+        }
+    }
+    __syncthreads();
+
+    // ---- (ii) one softmax per query: warp g owns query g ---------------------------------------
+    for (int g = warp; g < G; g += NW) {
+        float *wg = w + g * wstride;
+        float m = -INFINITY;
+        for (int s = lane; s <= cnt; s += 32) m = fmaxf(m, wg[s]);
+        m = warp_max(m);
+        float l = 0.f;
+        for (int s = lane; s <= cnt; s += 32) {
+            const float e = expf(wg[s] - m);
+            wg[s] = e;
+            l += e;
+        }
+        l = warp_sum(l);
+        const float inv = 1.f / l;
+        for (int s = lane; s <= cnt; s += 32) wg[s] *= inv;       // probabilities from here on
+    }
+    __syncthreads();
+
+    // ---- (iii) out_g = sum_slot a_g[slot] V[slot] + a_g[self] v_new -----------------------------
+    float acc[kMaxGroup][VEC];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[g][e] = 0.f;
+    for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
+        uint4 raw[kUnroll];
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int s = s0 + x * NW * RPW + rsel;
+            raw[x] = make_uint4(0u, 0u, 0u, 0u);
+            if (s <= cnt)
+                raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? Vu + (size_t)s * D : vnu) + sub * VEC);
+        }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) {
+            const int s = s0 + x * NW * RPW + rsel;
+            if (s <= cnt) {
+                float vf[VEC];
+                Elem<T>::unpack(raw[x], vf);
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g) {
+                    if (g < G) {
+                        const float a = w[g * wstride + s];
+#pragma unroll
+                        for (int e = 0; e < VEC; ++e) acc[g][e] = fmaf(a, vf[e], acc[g][e]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+        if (g < G) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+                float v = acc[g][e];
+#pragma unroll
+                for (int o = LPR; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);   // over rsel
+                if (rsel == 0) part[((size_t)warp * G + g) * D + sub * VEC + e] = v;
+            }
+        }
+    }
+    __syncthreads();
+    for (int x = tid; x < G * D; x += kGroupThreads) {
+        float o = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < NW; ++wv) o += part[(size_t)wv * G * D + x];
+        out[(size_t)u * G * D + x] = Elem<T>::from_float(o);
+    }
+
+    // ---- (iv) S <- alpha*S + sum_g a_g ; candidates for eviction ---------------------------------
+    const bool full = cnt >= M;
+    const int newest_evictable = p - c.R;
+    unsigned long long best = ~0ull;
+    int best_slot = -1;
+    for (int s = tid; s < cnt; s += kGroupThreads) {
+        float gain = 0.f;
+        for (int g = 0; g < G; ++g) gain += w[g * wstride + s];
+        const float sn = fmaf(alpha, Su[s], gain);
+        Su[s] = sn;
+        const int ps = posu[s];
+        if (full && ps <= newest_evictable) {
+            const unsigned long long key = ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
+            if (key < best) { best = key; best_slot = s; }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+        if (ob < best) { best = ob; best_slot = os; }
+    }
+    if (lane == 0) { red_key[warp] = best; red_slot[warp] = best_slot; }
+    __syncthreads();
+
+    // ---- (v) eviction and in-place insert, (vi) length ------------------------------------------
+    float s_new = 0.f;
+    for (int g = 0; g < G; ++g) s_new += w[g * wstride + cnt];
+    if (tid == 0) {
+        int target = full ? -2 : cnt;
+        if (full) {
+            unsigned long long gb = red_key[0];
+            int gs = red_slot[0];
+            for (int x = 1; x < NW; ++x)
+                if (red_key[x] < gb) { gb = red_key[x]; gs = red_slot[x]; }
+            const unsigned long long self_key = ((unsigned long long)__float_as_uint(s_new) << 32) | (unsigned)p;
+            if (gs >= 0 && (c.R > 0 || gb < self_key)) target = gs;
+        }
+        s_target = target;
+    }
+    __syncthreads();
+    const int target = s_target;
+    if (target >= 0) {
+        if (tid < LPR)
+            *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
+                *reinterpret_cast<const uint4 *>(knu + tid * VEC);
+        else if (tid < 2 * LPR)
+            *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
+                *reinterpret_cast<const uint4 *>(vnu + (tid - LPR) * VEC);
+    }
+    if (tid == 0) {
+        if (target >= 0) {
+            Su[target] = s_new;
+            posu[target] = p;
+        }
+        if (!full) c.count[u] = cnt + 1;
+        c.len[u] = p + 1;
+        evicted[u] = full ? target : -1;
+    }
+}
+
+template <typename T, int D>
+cudaError_t launch_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                         const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    const size_t wstride = ((size_t)c.M + 1 + 3) & ~(size_t)3;
+    const size_t smem = ((size_t)G * wstride + (size_t)(kGroupThreads / 32) * G * D) * sizeof(float);
+    if (smem > 220 * 1024) return cudaErrorInvalidValue;
+    auto kern = decode_step_group_kernel<T, D>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<c.U, kGroupThreads, smem, s>>>(c, G, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
+                                           static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_group_sum(const float *per_head, float *out, int G, int n, size_t units, cudaStream_t s)
+{
+    const size_t total = units * (size_t)n;
+    const unsigned grid = (unsigned)std::min<size_t>((total + 255) / 256, 148 * 16);
+    group_sum_kernel<<<grid, 256, 0, s>>>(per_head, out, G, n, total);
+    count_launch();
+    return cudaGetLastError();
+}
+
+size_t decode_group_smem_bytes(int M, int G, int d)
+{
+    const size_t wstride = ((size_t)M + 1 + 3) & ~(size_t)3;
+    return ((size_t)G * wstride + (size_t)(kGroupThreads / 32) * G * d) * sizeof(float);
+}
+
+cudaError_t launch_decode_step_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                                     const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    if (G < 1 || G > kMaxGroup) return cudaErrorInvalidValue;
+#define A2SF_DISPATCH(T)                                                                  \
+    (c.d == 64 ? launch_group<T, 64>(c, G, alpha, q, k_new, v_new, out, evicted, s)        \
+               : launch_group<T, 128>(c, G, alpha, q, k_new, v_new, out, evicted, s))
+    switch (c.dtype) {
+    case A2SF_F32: return A2SF_DISPATCH(float);
+    case A2SF_BF16: return A2SF_DISPATCH(__nv_bfloat16);
+    default: return A2SF_DISPATCH(__half);
+    }
+#undef A2SF_DISPATCH
+}
+
+}  // namespace a2sf

@@ -348,6 +348,78 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     cache.close()
 
 
+# ---- grouped query heads: several query heads on one K/V head and one cache ---------------------
+@pytest.mark.parametrize("name,kw,G", [
+    ("llama2_13b", dict(B=1, H=2, n=700, budget=96, recent=48, steps=30), 4),     # bf16, tensor-core passes
+    ("opt_6p7b", dict(B=2, H=1, n=300, budget=64, recent=0, steps=40, alpha=0.7), 8),   # fp16, all selective
+    ("tiny_fp32", dict(H=3, n=150, steps=24), 2),                                  # fp32 d = 64, CUDA cores
+    ("llama2_7b", dict(H=2, n=40, budget=64, recent=32, steps=40), 3),             # appends, then evicts
+])
+def test_grouped_query_heads_against_the_oracle(name, kw, G):
+    import oracle
+    from parity_util import ParityReport, TIE_RTOL, check_kept, check_out, check_scores, to_f64
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    T = w.steps
+    # query heads come from a workload with H*G heads; K/V heads from the workload itself
+    wq = w.scaled(H=w.H * G)
+    q = wl.make_prompt(wq, device="cuda")[0]
+    _, k, v = wl.make_prompt(w, device="cuda")
+    dq = wl.make_decode(wq, device="cuda")[0]                     # [T, B, H*G, d]
+    _, dk, dv = wl.make_decode(w, device="cuda")                  # [T, B, H, d]
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    out, S, kept, lse = a2sf.a2sf_prefill_group(p, G, q, k, v)
+    torch.cuda.synchronize()
+    U, n, d = w.units, w.n, w.d
+    Qo = to_f64(q).reshape(U, G, n, d)
+    Ko, Vo = to_f64(k).reshape(U, n, d), to_f64(v).reshape(U, n, d)
+    ref = oracle.group_prefill(Qo, Ko, Vo, w.scale, w.alpha, w.budget, w.recent, nthreads=oracle.host_threads())
+    rep = ParityReport()
+    check_out(to_f64(out).reshape(U, G, n, d), ref["out"], w.dtype, rep, "grouped prefill out")
+    assert np.abs(to_f64(lse).reshape(U, G, n) - ref["lse"]).max() <= 1e-4 * max(1.0, np.abs(ref["lse"]).max())
+    check_scores(to_f64(S).reshape(U, n), ref["S"], rep, "grouped prefill scores")
+    kg = kept.cpu().numpy().reshape(U, -1)
+    for u in range(U):
+        check_kept(kg[u], ref["kept"][u], ref["S"][u], n, w.budget, w.recent)
+
+    cache = a2sf.Cache(p)
+    cache.a2sf_cache_load(k, v, S, kept)
+    oc = oracle.GroupCache(U, d, w.budget, w.recent, w.scale)
+    oc.load(Ko, Vo, ref["S"], kg)
+    o_t = torch.empty((w.B, w.H * G, d), dtype=q.dtype, device="cuda")
+    e_t = torch.empty((w.B, w.H), dtype=torch.int32, device="cuda")
+    excused = evictions = 0
+    for t in range(T):
+        cache.a2sf_decode_step_group(G, w.alpha, dq[t].contiguous(), dk[t].contiguous(), dv[t].contiguous(),
+                                     o_t, e_t)
+        torch.cuda.synchronize()
+        ev = e_t.cpu().numpy().reshape(U)
+        force = np.where(ev == -1, -3, ev).astype(np.int32)
+        o_ref, info, sc = oc.step_group(to_f64(dq[t]).reshape(U, G, d), to_f64(dk[t]).reshape(U, d),
+                                        to_f64(dv[t]).reshape(U, d), w.alpha, force=force)
+        for u in range(U):
+            if info[u, 1] == -1:
+                assert ev[u] == -1
+                continue
+            evictions += 1
+            if ev[u] != info[u, 1]:
+                assert abs(sc[u, 0] - sc[u, 1]) <= TIE_RTOL * max(abs(sc[u, 0]), abs(sc[u, 1]))
+                excused += 1
+        check_out(to_f64(o_t).reshape(U, G, d), o_ref, w.dtype, rep, f"grouped step {t} out")
+    st = cache.a2sf_cache_export()
+    torch.cuda.synchronize()
+    cnt = st["count"].cpu().numpy().reshape(U)
+    np.testing.assert_array_equal(cnt, oc.count)
+    pos, Sg = st["pos"].cpu().numpy().reshape(U, -1), to_f64(st["scores"]).reshape(U, -1)
+    for u in range(U):
+        np.testing.assert_array_equal(pos[u, :cnt[u]], oc.pos[u, :cnt[u]])
+        check_scores(Sg[u, :cnt[u]], oc.S[u, :cnt[u]], rep, "grouped cache scores")
+    assert excused <= max(2, evictions // 200) and a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+    print(f"\n[grouped] {w.name} G={G}: units={U} n={n} steps={T} evictions={evictions} excused={excused} "
+          f"max_out={rep.max_out_err:.3g} max_score_rel={rep.max_score_rel:.3g}")
+
+
 # ---- similarity with the ideal mask ----------------------------------------------------------------
 @pytest.mark.parametrize("name,kw", [
     ("tiny_fp32", dict()),                                                     # fp32, d = 64
