@@ -436,6 +436,24 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         }
         sh->abort_flag = 0;
         fence_mbar_init();
+        // The first tiles are requested here, before the tensor-memory allocation and the
+        // CTA-wide barrier: their latency (about 5000 clocks until Q and K arrive) is the
+        // longest item of a CTA's start-up.
+        prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+        mbar_arrive_expect_tx(&sh->q_full, hasB ? 2 * kTileBytes : kTileBytes);
+        tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rbA * kBlk, h, b);
+        tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rbA * kBlk, h, b);
+        if (hasB) {
+            tma_load_4d(Qs + kTileBytes, &tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
+            tma_load_4d(Qs + kTileBytes + kHalfBytes, &tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
+        }
+        const int hk0 = h / a.G;
+        mbar_arrive_expect_tx(&sh->k_full[0], kTileBytes);
+        tma_load_4d(Ks, &tmap_k, &sh->k_full[0], 0, 0, hk0, b);
+        tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full[0], 64, 0, hk0, b);
+        mbar_arrive_expect_tx(&sh->v_full[0], kTileBytes);
+        tma_load_4d(Vs, &tmap_v, &sh->v_full[0], 0, 0, hk0, b);
+        tma_load_4d(Vs + kHalfBytes, &tmap_v, &sh->v_full[0], 64, 0, hk0, b);
     }
     if (warp == 1) {
         tmem_alloc(&sh->tmem_base, 512);
@@ -456,17 +474,10 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     if (warp == 0) {
         // ---- TMA producer -------------------------------------------------------------
         if (lane == 0) {
-            prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
-            mbar_arrive_expect_tx(&sh->q_full, hasB ? 2 * kTileBytes : kTileBytes);
-            tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rbA * kBlk, h, b);
-            tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rbA * kBlk, h, b);
-            if (hasB) {
-                tma_load_4d(Qs + kTileBytes, &tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
-                tma_load_4d(Qs + kTileBytes + kHalfBytes, &tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
-            }
+            // Q and the first K and V tiles were requested during set-up
             const int hk = h / a.G;                   // the K/V head this query head reads
-            int k_issued = 0, v_issued = 0;
-            for (int t = 0; t < nt; ++t) {
+            int k_issued = 1, v_issued = 1;
+            for (int t = 1; t < nt; ++t) {
                 const int ks = t % kKStages, vs = t % kVStages;
                 if (!wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
