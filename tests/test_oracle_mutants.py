@@ -129,3 +129,69 @@ def test_mutant_is_caught(tmp_path, name):
     lib = _build(tmp_path, name, SRC.replace(old, new, 1))
     with pytest.raises(AssertionError):
         run_pins(lib)
+
+
+# ---- the numpy parts of the oracle (streamed prompt, ideal similarity, grouped heads) ---------------
+PY_SRC = Path(oracle.__file__).read_text()
+
+PY_MUTANTS = {
+    "ideal_keeps_the_smallest": ("order = np.lexsort((np.arange(m), -s_row))", "order = np.lexsort((np.arange(m), s_row))"),
+    "ideal_tie_prefers_higher_position": ("order = np.lexsort((np.arange(m), -s_row))",
+                                          "order = np.lexsort((-np.arange(m), -s_row))"),
+    "ideal_row_not_normalised": ("    p[order] = w / w.sum()\n    return p", "    p[order] = w\n    return p"),
+    "ideal_keeps_budget_not_budget_plus_one": ("ideal = ideal_row(s_row, M + 1)", "ideal = ideal_row(s_row, M)"),
+    "policy_row_without_the_token_itself": ("seen = np.append(cache.pos[u, :cache.count[u]], i)",
+                                            "seen = cache.pos[u, :cache.count[u]] if cache.count[u] else np.array([i])"),
+    "cosine_without_norms": ("cos[u, i] = (meth @ ideal) / np.sqrt((meth @ meth) * (ideal @ ideal))",
+                             "cos[u, i] = (meth @ ideal)"),
+    "streamed_rows_use_the_previous_key": ("o, info[i], sc[i] = cache.step(Q[:, i], K[:, i], V[:, i], alpha,\n                                        force=None if force is None else force[i], nthreads=nthreads)\n        out[:, i] = o\n    return out, info, sc, cache",
+                                           "o, info[i], sc[i] = cache.step(Q[:, i], K[:, max(i - 1, 0)], V[:, i], alpha,\n                                        force=None if force is None else force[i], nthreads=nthreads)\n        out[:, i] = o\n    return out, info, sc, cache"),
+    "group_mean_instead_of_sum": ("                gain += a\n", "                gain += a / G\n"),
+    "group_decay_after_add": ("self.S[u, :cnt] = alpha * self.S[u, :cnt] + gain[:cnt]",
+                              "self.S[u, :cnt] = alpha * (self.S[u, :cnt] + gain[:cnt])"),
+    "group_self_score_from_one_head": ("            s_new = gain[cnt]\n", "            s_new = a[cnt]\n"),
+    "group_recent_window_off_by_one": ("if self.pos[u, s] <= p - self.R]", "if self.pos[u, s] < p - self.R]"),
+    "group_prefill_keeps_one_head": ('        S += r["S"][:, 0]\n', '        S = r["S"][:, 0].copy()\n'),
+}
+
+
+def _py_pins(pins):
+    pins.test_ideal_row_is_a_top_k_softmax()
+    pins.test_similarity_is_one_while_nothing_is_pruned_and_bounded_after()
+    pins.test_streamed_prompt_without_eviction_is_the_dense_prefill()
+    pins.test_streamed_prompt_with_recent_equal_budget_is_a_sliding_window()
+    pins.test_streamed_prompt_matches_a_mask_matrix_construction(6, 2, 0.5)
+    pins.test_group_of_one_is_the_single_head_step()
+    pins.test_group_scores_are_the_sum_of_the_heads_attention()
+    pins.test_group_eviction_follows_the_summed_score()
+
+
+def _load_py(tmp_path, name, src):
+    import importlib.util
+
+    real = Path(oracle.__file__).resolve().parent
+    src = src.replace("_HERE = Path(__file__).resolve().parent", f"_HERE = Path({str(real)!r})")
+    f = tmp_path / f"oracle_{name}.py"
+    f.write_text(src)
+    spec = importlib.util.spec_from_file_location(f"oracle_{name}", f)
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def test_unmodified_python_oracle_passes_its_pins(tmp_path, monkeypatch):
+    import test_oracle_pins as pins
+
+    monkeypatch.setattr(pins, "oracle", _load_py(tmp_path, "clean", PY_SRC))
+    _py_pins(pins)
+
+
+@pytest.mark.parametrize("name", sorted(PY_MUTANTS))
+def test_python_oracle_mutant_is_caught(name, tmp_path, monkeypatch):
+    import test_oracle_pins as pins
+
+    old, new = PY_MUTANTS[name]
+    assert PY_SRC.count(old) == 1, f"mutation site of {name} not found exactly once"
+    monkeypatch.setattr(pins, "oracle", _load_py(tmp_path, name, PY_SRC.replace(old, new)))
+    with pytest.raises(AssertionError):
+        _py_pins(pins)
