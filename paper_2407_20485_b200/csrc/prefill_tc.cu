@@ -343,7 +343,6 @@ struct AttnArgs {
     int G;                // query heads per key/value head
     float sl2;            // scale * log2(e)
     const int *v_flag;    // bf16 storage: 0 = the fp16 copy of V is exact, 1 = it is not
-    int run_if_flag;      // this launch works only when *v_flag equals this value
 };
 
 struct AttnShared {
@@ -373,13 +372,12 @@ template <> __device__ __forceinline__ uint32_t pack2<__half>(float a, float b)
 }
 
 // PvHalf (bf16 storage only): the P V product runs in fp16 -- P is rounded to fp16 (11
-// significand bits, one term) and V comes from an fp16 copy made beforehand.  The launch works
-// only if that copy is exact (*v_flag == 0); otherwise the plain bf16 launch, which writes P as
-// two bf16 terms, does the work.
+// significand bits, one term) and V comes from an fp16 copy made beforehand.  That form is valid
+// only if the copy is exact; otherwise the plain bf16 form, which writes P as two bf16 terms,
+// does the work (attn_pass_bf16_auto picks one of the two on the device).
 template <typename T, bool PvHalf>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-             const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
+__device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUtensorMap *tmap_k,
+                                          const CUtensorMap *tmap_v, const AttnArgs &a)
 {
     // once any CTA has given up on a wait, the rest of the grid drains without working
     extern __shared__ __align__(1024) uint8_t attn_smem[];
@@ -387,7 +385,6 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         int skip = 0;
         if (threadIdx.x == 0) {
             skip = *reinterpret_cast<volatile int *>(&g_tc_status);
-            if (a.v_flag && (*a.v_flag != 0) != (a.run_if_flag != 0)) skip = 1;   // the other launch's job
             if (smem_u32(attn_smem) & 1023u) {           // the swizzled tiles need this alignment
                 g_tc_status = A2SF_ERR_CUDA;
                 skip = 1;
@@ -439,21 +436,21 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
         // The first tiles are requested here, before the tensor-memory allocation and the
         // CTA-wide barrier: their latency (about 5000 clocks until Q and K arrive) is the
         // longest item of a CTA's start-up.
-        prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+        prefetch_tmap(tmap_q); prefetch_tmap(tmap_k); prefetch_tmap(tmap_v);
         mbar_arrive_expect_tx(&sh->q_full, hasB ? 2 * kTileBytes : kTileBytes);
-        tma_load_4d(Qs, &tmap_q, &sh->q_full, 0, rbA * kBlk, h, b);
-        tma_load_4d(Qs + kHalfBytes, &tmap_q, &sh->q_full, 64, rbA * kBlk, h, b);
+        tma_load_4d(Qs, tmap_q, &sh->q_full, 0, rbA * kBlk, h, b);
+        tma_load_4d(Qs + kHalfBytes, tmap_q, &sh->q_full, 64, rbA * kBlk, h, b);
         if (hasB) {
-            tma_load_4d(Qs + kTileBytes, &tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
-            tma_load_4d(Qs + kTileBytes + kHalfBytes, &tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
+            tma_load_4d(Qs + kTileBytes, tmap_q, &sh->q_full, 0, rbB * kBlk, h, b);
+            tma_load_4d(Qs + kTileBytes + kHalfBytes, tmap_q, &sh->q_full, 64, rbB * kBlk, h, b);
         }
         const int hk0 = h / a.G;
         mbar_arrive_expect_tx(&sh->k_full[0], kTileBytes);
-        tma_load_4d(Ks, &tmap_k, &sh->k_full[0], 0, 0, hk0, b);
-        tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full[0], 64, 0, hk0, b);
+        tma_load_4d(Ks, tmap_k, &sh->k_full[0], 0, 0, hk0, b);
+        tma_load_4d(Ks + kHalfBytes, tmap_k, &sh->k_full[0], 64, 0, hk0, b);
         mbar_arrive_expect_tx(&sh->v_full[0], kTileBytes);
-        tma_load_4d(Vs, &tmap_v, &sh->v_full[0], 0, 0, hk0, b);
-        tma_load_4d(Vs + kHalfBytes, &tmap_v, &sh->v_full[0], 64, 0, hk0, b);
+        tma_load_4d(Vs, tmap_v, &sh->v_full[0], 0, 0, hk0, b);
+        tma_load_4d(Vs + kHalfBytes, tmap_v, &sh->v_full[0], 64, 0, hk0, b);
     }
     if (warp == 1) {
         tmem_alloc(&sh->tmem_base, 512);
@@ -481,13 +478,13 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
                 const int ks = t % kKStages, vs = t % kVStages;
                 if (!wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
-                tma_load_4d(Ks + ks * kTileBytes, &tmap_k, &sh->k_full[ks], 0, t * kBlk, hk, b);
-                tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, &tmap_k, &sh->k_full[ks], 64, t * kBlk, hk, b);
+                tma_load_4d(Ks + ks * kTileBytes, tmap_k, &sh->k_full[ks], 0, t * kBlk, hk, b);
+                tma_load_4d(Ks + ks * kTileBytes + kHalfBytes, tmap_k, &sh->k_full[ks], 64, t * kBlk, hk, b);
                 k_issued = t + 1;
                 if (!wait(&sh->v_empty[vs], ((t / kVStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->v_full[vs], kTileBytes);
-                tma_load_4d(Vs + vs * kTileBytes, &tmap_v, &sh->v_full[vs], 0, t * kBlk, hk, b);
-                tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, &tmap_v, &sh->v_full[vs], 64, t * kBlk, hk, b);
+                tma_load_4d(Vs + vs * kTileBytes, tmap_v, &sh->v_full[vs], 0, t * kBlk, hk, b);
+                tma_load_4d(Vs + vs * kTileBytes + kHalfBytes, tmap_v, &sh->v_full[vs], 64, t * kBlk, hk, b);
                 v_issued = t + 1;
             }
             if (*abort_flag) {
@@ -707,6 +704,29 @@ attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__
     if (threadIdx.x == 0 && sh->abort_flag) g_tc_status = A2SF_ERR_TIMEOUT;
 }
 
+template <typename T, bool PvHalf>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+             const __grid_constant__ CUtensorMap tmap_v, AttnArgs a)
+{
+    attn_body<T, PvHalf>(&tmap_q, &tmap_k, &tmap_v, a);
+}
+
+// bf16 storage with an fp16 copy of V in the workspace: one launch, and the flag written by the
+// conversion kernel decides on the device which form of the P V product runs -- fp16 P with the
+// fp16 copy when the copy is exact, two bf16 terms with the original V when it is not.
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_pass_bf16_auto(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_v_half,
+                    AttnArgs a)
+{
+    const bool exact = *a.v_flag == 0;
+    AttnArgs b = a;
+    b.v_flag = nullptr;
+    if (exact) attn_body<__nv_bfloat16, true>(&tmap_q, &tmap_k, &tmap_v_half, b);
+    else       attn_body<__nv_bfloat16, false>(&tmap_q, &tmap_k, &tmap_v, b);
+}
+
 // fp16 copy of a bf16 V tensor, contiguous [U][n][d], for the PvHalf attention launch.  A bf16
 // value converts exactly when its magnitude is within fp16's range (magnitudes below 2^-17 lose
 // at most 2^-25 absolutely, which is immaterial); any value beyond 65504, infinite or NaN raises
@@ -803,7 +823,7 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
         const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
         attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, false>, attr, (int)kAttnSmemBytes);
         if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, true>, attr, (int)kAttnSmemBytes);
+            attr_err = cudaFuncSetAttribute(attn_pass_bf16_auto, attr, (int)kAttnSmemBytes);
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(attn_pass_tc<__half, false>, attr, (int)kAttnSmemBytes);
     });
@@ -813,7 +833,7 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
     aa.n = a.n; aa.H = a.H; aa.G = a.G;
     aa.sl2 = a.scale * kLog2e;
-    aa.v_flag = nullptr; aa.run_if_flag = 0;
+    aa.v_flag = nullptr;
     const int npairs = ((a.n + kBlk - 1) / kBlk + 1) / 2;
     const dim3 grid((unsigned)((size_t)a.B * a.H * npairs));
     if (dtype == A2SF_F16) {
@@ -826,8 +846,8 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
         count_launch();
         return cudaGetLastError();
     }
-    // bf16: make the fp16 copy of V, then launch both forms of the pass; the flag written by
-    // the copy decides on the device which of the two does the work (no host round trip)
+    // bf16: make the fp16 copy of V, then one launch that picks the form of the P V product on
+    // the device from the flag the copy wrote (no host round trip)
     cudaError_t e = cudaMemsetAsync(a.v_flag, 0, sizeof(int), s);
     if (e != cudaSuccess) return e;
     const size_t chunks = (size_t)a.B * Hkv * a.n * (kD / 8);
@@ -840,12 +860,7 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     CUtensorMap mvh;
     if (!make_tile_map(&mvh, A2SF_F16, a.v_half, a, Hkv, contig)) return cudaErrorInvalidValue;
     aa.v_flag = a.v_flag;
-    aa.run_if_flag = 0;
-    attn_pass_tc<__nv_bfloat16, true><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mvh, aa);
-    count_launch();
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    aa.run_if_flag = 1;
-    attn_pass_tc<__nv_bfloat16, false><<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, aa);
+    attn_pass_bf16_auto<<<grid, kAttnThreads, kAttnSmemBytes, s>>>(mq, mk, mv, mvh, aa);
     count_launch();
     return cudaGetLastError();
 }
