@@ -186,15 +186,19 @@ def run_ours(args):
 
     # ---- the two prefill passes apart: the scoring pass + selection run alone from the saved lse
     # (a2sf_rescore); the attention pass is the rest of the prefill time measured above
-    er = cuda_events(2)
+    er = cuda_events(3)
     a2sf.a2sf_rescore(p, q, k, lse, scores=scores, kept_idx=kept)
     reps_r = 5
     er[0].record()
     for _ in range(reps_r):
         a2sf.a2sf_rescore(p, q, k, lse, scores=scores, kept_idx=kept)
     er[1].record()
+    for _ in range(reps_r):       # the whole prefill under the same (short-run) clocks
+        a2sf.a2sf_prefill(p, q, k, v, out=out, scores=scores, kept_idx=kept, lse=lse, workspace=ws)
+    er[2].record()
     torch.cuda.synchronize()
     rescore_ms = er[0].elapsed_time(er[1]) / reps_r
+    prefill_short_ms = er[1].elapsed_time(er[2]) / reps_r
 
     # ---- separate line: the scoring pass without the rows whose forgetting weight is exactly
     # zero in fp32 (bit-identical scores, less work; NOT part of the headline step above)
@@ -317,10 +321,12 @@ def run_ours(args):
                     "passes": {
                         "scores_and_selection_ms": rescore_ms,
                         "scores_tflops": U * flops["pass2"] / (rescore_ms * 1e-3) / 1e12,
-                        "attention_ms": prefill_ms / K - rescore_ms,
-                        "attention_tflops": U * flops["pass1"] / ((prefill_ms / K - rescore_ms) * 1e-3) / 1e12,
-                        "note": "this rank; attention = prefill - (scores + selection), includes the "
-                                "fp16 copy of V for bf16 storage"}},
+                        "prefill_ms": prefill_short_ms,
+                        "attention_ms": prefill_short_ms - rescore_ms,
+                        "attention_tflops": U * flops["pass1"] / ((prefill_short_ms - rescore_ms) * 1e-3) / 1e12,
+                        "note": "this rank, 5 back-to-back repetitions after the timed region (shorter "
+                                "run, higher clocks than inside it); attention = prefill - (scores + "
+                                "selection), includes the fp16 copy of V for bf16 storage"}},
         "roofline": {"kernel": "decode_step_stream_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
