@@ -485,6 +485,36 @@ def test_several_tokens_in_one_call_equal_single_steps():
         assert torch.equal(s1[key], s2[key]), key
 
 
+def test_graphed_steps_helper_continues_a_cache_like_single_calls():
+    from paper_2407_20485_b200 import binding as a2sf
+    from paper_2407_20485_b200.graphs import GraphedSteps
+
+    w = W["opt_6p7b"].scaled(B=1, H=4, n=260, steps=12)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    dq, dk, dv = wl.make_decode(w, device="cuda")
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    _, S, kept, _ = a2sf.a2sf_prefill(p, q, k, v)
+    a, b = a2sf.Cache(p), a2sf.Cache(p)
+    a.a2sf_cache_load(k, v, S, kept)
+    b.a2sf_cache_load(k, v, S, kept)
+    T = 4                                                   # three replays of four steps
+    o1 = torch.empty((w.steps, w.B, w.H, w.d), dtype=q.dtype, device="cuda")
+    e1 = torch.empty((w.steps, w.B, w.H), dtype=torch.int32, device="cuda")
+    for t in range(w.steps):
+        a.a2sf_decode_step(w.alpha, dq[t], dk[t], dv[t], o1[t], e1[t])
+    bq, bk, bv = dq[:T].clone(), dk[:T].clone(), dv[:T].clone()
+    g = GraphedSteps(b, w.alpha, bq, bk, bv)
+    for r in range(w.steps // T):
+        bq.copy_(dq[r * T:(r + 1) * T]); bk.copy_(dk[r * T:(r + 1) * T]); bv.copy_(dv[r * T:(r + 1) * T])
+        out, ev = g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, o1[r * T:(r + 1) * T]) and torch.equal(ev, e1[r * T:(r + 1) * T])
+    sa, sb = a.a2sf_cache_export(), b.a2sf_cache_export()
+    torch.cuda.synchronize()
+    for key in ("scores", "pos", "count", "len", "k", "v"):
+        assert torch.equal(sa[key], sb[key]), key
+
+
 # ---- scoring pass that leaves out rows whose forgetting weight is exactly zero ------------------
 @pytest.mark.parametrize("name,kw,alphas", [
     ("llama2_13b", dict(B=1, H=3, n=1100), [0.5, 0.9, 0.0, 1.0, 0.3]),      # tensor-core pass
