@@ -96,6 +96,16 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v)
 // ---- host-side launch bookkeeping -------------------------------------------
 void count_launch(int n = 1);
 
+// Kernel attributes, symbol addresses and SM counts belong to a device: state that is set up
+// once is kept per device, indexed by the current one.
+constexpr int kMaxDevices = 64;
+inline int current_device_index()
+{
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= kMaxDevices) d = 0;
+    return d;
+}
+
 // ---- kernel launchers (one per translation unit) -----------------------------
 struct PrefillArgs {
     const void *q, *k, *v;

@@ -21,12 +21,13 @@ namespace {
 
 int *decode_status_word()
 {
-    static int *ptr = nullptr;
-    if (!ptr) {
+    static int *ptr[kMaxDevices] = {};
+    const int dev = current_device_index();
+    if (!ptr[dev]) {
         void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_decode_status) == cudaSuccess) ptr = static_cast<int *>(p);
+        if (cudaGetSymbolAddress(&p, g_decode_status) == cudaSuccess) ptr[dev] = static_cast<int *>(p);
     }
-    return ptr;
+    return ptr[dev];
 }
 
 constexpr int kDecodeThreads = 256;
@@ -738,25 +739,23 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const float *alpha_ve
     if (stages > kMaxStreamStages) stages = kMaxStreamStages;
     const size_t smem = fixed + (size_t)stages * kChunkBytes;
     auto kern = decode_step_stream_kernel<T, D>;
-    static int num_sms = 0;
-    if (num_sms == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    }
+    static int sm_count[kMaxDevices] = {};
+    const int dev = current_device_index();
+    if (sm_count[dev] == 0) cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    const int num_sms = sm_count[dev];
     // Few units with long caches would leave most SMs idle: split each unit over a cluster.
     if (c.M >= kSplitMinBudget && c.U * 2 <= num_sms) {
         int cs = 2;
         while (cs < 8 && c.U * cs * 2 <= 2 * num_sms) cs *= 2;
         return launch_split<T, D>(c, cs, alpha, alpha_vec, q, k_new, v_new, out, evicted, s);
     }
-    static cudaError_t attr_err = cudaSuccess;
-    static size_t attr_smem = 0;
-    if (smem > attr_smem) {
-        attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_smem = smem;
+    static cudaError_t attr_err[kMaxDevices] = {};
+    static size_t attr_smem[kMaxDevices] = {};
+    if (smem > attr_smem[dev]) {
+        attr_err[dev] = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        attr_smem[dev] = smem;
     }
-    if (attr_err != cudaSuccess) return attr_err;
+    if (attr_err[dev] != cudaSuccess) return attr_err[dev];
     int *status = decode_status_word();
     if (!status) return cudaErrorUnknown;
     const int grid = c.U < ctas_per_sm * num_sms ? c.U : ctas_per_sm * num_sms;

@@ -817,17 +817,17 @@ cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_
     if (!make_tile_map(&mq, dtype, a.q, a, a.H, a.st) || !make_tile_map(&mk, dtype, a.k, a, Hkv, a.st_kv) ||
         !make_tile_map(&mv, dtype, a.v, a, Hkv, a.st_kv))
         return cudaErrorInvalidValue;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
+    static std::once_flag once[kMaxDevices];
+    static cudaError_t attr_errs[kMaxDevices] = {};
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
         const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-        attr_err = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, false>, attr, (int)kAttnSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_pass_bf16_auto, attr, (int)kAttnSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(attn_pass_tc<__half, false>, attr, (int)kAttnSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(attn_pass_tc<__nv_bfloat16, false>, attr, (int)kAttnSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_pass_bf16_auto, attr, (int)kAttnSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_pass_tc<__half, false>, attr, (int)kAttnSmemBytes);
+        attr_errs[dev] = e;
     });
-    if (attr_err != cudaSuccess) return attr_err;
+    if (attr_errs[dev] != cudaSuccess) return attr_errs[dev];
     AttnArgs aa;
     aa.out = a.out; aa.lse = a.lse;
     aa.st_b = a.st.b; aa.st_h = a.st.h; aa.st_t = a.st.t;
@@ -871,13 +871,14 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     if (!make_tile_map(&mq, dtype, a.q, a, a.H, a.st) ||
         !make_tile_map(&mk, dtype, a.k, a, a.H / a.G, a.st_kv))
         return cudaErrorInvalidValue;
-    static std::once_flag once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(once, [] {
-        attr_err = cudaFuncSetAttribute(score_pass_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)kScoreSmemBytes);
+    static std::once_flag once[kMaxDevices];
+    static cudaError_t attr_errs[kMaxDevices] = {};
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
+        attr_errs[dev] = cudaFuncSetAttribute(score_pass_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)kScoreSmemBytes);
     });
-    if (attr_err != cudaSuccess) return attr_err;
+    if (attr_errs[dev] != cudaSuccess) return attr_errs[dev];
     ScoreArgs sa;
     sa.lse = a.lse; sa.scores = a.scores; sa.n = a.n; sa.H = a.H; sa.G = a.G;
     sa.sl2 = a.scale * kLog2e;
