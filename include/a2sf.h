@@ -52,8 +52,11 @@ typedef enum {
 /* Shape and policy of a call.  `scale` = 0 selects 1/sqrt(d).  `alpha` is the
  * forgetting factor of Eq. 5; the paper states 0 < alpha < 1 and also runs
  * alpha = 0 (Sec. 4.4); alpha = 1 is the plain accumulative score of H2O (Eq. 4).
- * Accepted: 0 <= alpha <= 1 with alpha^0 = 1.  budget >= 1, 0 <= recent <= budget,
- * d in {64, 128}. */
+ * Accepted: 0 <= alpha <= 1 with alpha^0 = 1.  1 <= budget <= A2SF_MAX_BUDGET (one unit's
+ * logits of a generation step are held in one CTA's shared memory), 0 <= recent <= budget,
+ * d in {64, 128}.  Anything else: A2SF_ERR_INVALID_ARG, or A2SF_ERR_UNSUPPORTED for a dtype,
+ * head size or budget outside the supported set. */
+#define A2SF_MAX_BUDGET 49152
 typedef struct a2sf_params {
     int32_t B, H, d;
     int32_t dtype;               /* a2sf_dtype of q, k, v, out and the cache rows */

@@ -26,6 +26,7 @@ static int check_params(const a2sf_params *p)
     if (p->dtype != A2SF_F32 && p->dtype != A2SF_BF16 && p->dtype != A2SF_F16)
         return A2SF_ERR_UNSUPPORTED;
     if (p->d != 64 && p->d != 128) return A2SF_ERR_UNSUPPORTED;
+    if (p->budget > A2SF_MAX_BUDGET) return A2SF_ERR_UNSUPPORTED;
     if ((int64_t)p->B * p->H > 0x7fffffff) return A2SF_ERR_INVALID_ARG;
     if (p->flags & ~A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) return A2SF_ERR_INVALID_ARG;
     if (p->score_window < 0) return A2SF_ERR_INVALID_ARG;

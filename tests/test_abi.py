@@ -124,3 +124,14 @@ def test_score_window_bound_is_the_tail_of_the_geometric_series():
         tail = sum(a ** age for age in range(Wn, n)) if 0 < Wn < n else 0.0
         got = a2sf.a2sf_score_window_bound(alpha, n, Wn)
         assert abs(got - tail) <= 1e-12 * max(1.0, tail), (alpha, n, Wn, got, tail)
+
+
+def test_budget_beyond_the_documented_maximum_is_refused_on_the_host():
+    import torch
+    from paper_2407_20485_b200 import binding as a2sf
+
+    ok = a2sf.make_params(1, 1, 128, torch.bfloat16, 49152, 16, 0.5)
+    too_big = a2sf.make_params(1, 1, 128, torch.bfloat16, 49153, 16, 0.5)
+    assert a2sf.lib.a2sf_cache_bytes(ctypes.byref(ok)) > 0
+    assert a2sf.lib.a2sf_cache_bytes(ctypes.byref(too_big)) == 0
+    assert a2sf.lib.a2sf_prefill_workspace_bytes(ctypes.byref(too_big), 64) == 0

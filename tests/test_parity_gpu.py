@@ -72,6 +72,7 @@ def test_shrunken_configs(name, kw, alphas):
     dict(n=520, budget=512, recent=0, steps=20, dtype="fp16", d=128),    # all selective
     dict(n=100, budget=600, recent=10, steps=12),                        # most slices start empty
     dict(n=9, budget=1024, recent=1024, steps=6, dtype="bf16", d=128),   # fewer tokens than CTAs
+    dict(H=1, n=300, budget=49152, recent=64, steps=3, dtype="bf16", d=128),   # the largest budget
 ])
 def test_edge_cases(kw):
     w = W["tiny_fp32"].scaled(**kw)
