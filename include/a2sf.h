@@ -237,9 +237,10 @@ int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas,
                               const void *q, const void *k_new, const void *v_new,
                               void *out, int32_t *evicted_slot, void *cuda_stream);
 
-/* The same step with HOST buffers (pinned for asynchronous copies): q, k_new, v_new
- * are copied into staging rows inside the cache, the step runs, out and
- * evicted_slot are copied back.  Returns after the stream has drained. */
+/* The same step with HOST buffers.  Page-locked (pinned, mapped) buffers are read and written
+ * by the step kernel directly over the bus; for any other host memory q, k_new, v_new are
+ * copied into staging rows inside the cache, the step runs, out and evicted_slot are copied
+ * back.  Either way the call returns after the stream has drained, with the results in place. */
 int a2sf_decode_step_host(a2sf_cache *cache, float alpha,
                           const void *q_host, const void *k_new_host, const void *v_new_host,
                           void *out_host, int32_t *evicted_slot_host, void *cuda_stream);

@@ -545,6 +545,19 @@ int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas, const void
     return A2SF_OK;
 }
 
+// Device-side address of a pinned (page-locked, mapped) host buffer, or nullptr for anything
+// else (pageable memory, device memory, misaligned rows).
+static void *mapped_host_pointer(const void *host)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, host) != cudaSuccess) {
+        cudaGetLastError();                       // older drivers report pageable memory as an error
+        return nullptr;
+    }
+    if (at.type != cudaMemoryTypeHost || !at.devicePointer || !aligned(at.devicePointer, 16)) return nullptr;
+    return at.devicePointer;
+}
+
 int a2sf_decode_step_host(a2sf_cache *cache, float alpha, const void *q_host,
                           const void *k_new_host, const void *v_new_host, void *out_host,
                           int32_t *evicted_slot_host, void *cuda_stream)
@@ -552,6 +565,20 @@ int a2sf_decode_step_host(a2sf_cache *cache, float alpha, const void *q_host,
     if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !evicted_slot_host)
         return A2SF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // Pinned buffers are read and written by the step kernel itself, over the bus, while it
+    // streams the cache from device memory: five copies and their latencies less per step
+    // (about 1.3 KB per unit against the 270 KB of cache the same unit reads).
+    {
+        void *dq = mapped_host_pointer(q_host), *dk = mapped_host_pointer(k_new_host),
+             *dv = mapped_host_pointer(v_new_host), *dout = mapped_host_pointer(out_host),
+             *dev = mapped_host_pointer(evicted_slot_host);
+        if (dq && dk && dv && dout && dev) {
+            const int rc = a2sf_decode_step(cache, alpha, dq, dk, dv, dout, static_cast<int32_t *>(dev),
+                                            cuda_stream);
+            if (rc != A2SF_OK) return rc;
+            return cudaStreamSynchronize(s) == cudaSuccess ? A2SF_OK : A2SF_ERR_CUDA;
+        }
+    }
     const size_t U = cache->view.U;
     const size_t row = U * cache->p.d * elem_bytes(cache->p.dtype);
     if (cudaMemcpyAsync(cache->st_q, q_host, row, cudaMemcpyHostToDevice, s) != cudaSuccess ||
