@@ -288,19 +288,73 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const
     int32_t *dkept = reinterpret_cast<int32_t *>(base + 4 * tensor + align_up(U * n * 4));
     void *inner = base + 4 * tensor + align_up(U * n * 4) + align_up(U * m * 4);
 
-    if (cudaMemcpyAsync(dq, q_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dk, k_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(dv, v_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return A2SF_ERR_CUDA;
     const int64_t st = p->d, sh = (int64_t)n * p->d, sb = (int64_t)p->H * n * p->d;
-    rc = a2sf_prefill(p, n, dq, dk, dv, sb, sh, st, dout, dsc, dkept, nullptr, inner,
-                      prefill_ws_bytes(p, n), cuda_stream);
-    if (rc != A2SF_OK) return rc;
-    if (cudaMemcpyAsync(out_host, dout, tbytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(scores_host, dsc, U * n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(kept_idx_host, dkept, U * m * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return A2SF_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return A2SF_ERR_CUDA;
+    // Batch rows are independent, so the call is pipelined over chunks of them on two internal
+    // streams: while one chunk computes and its results travel back, the next chunk's inputs
+    // are already on their way in (the two copy directions and the kernels overlap).
+    const int chunks = p->B >= 2 ? (p->B < 8 ? p->B : 8) : 1;
+    if (chunks == 1) {
+        if (cudaMemcpyAsync(dq, q_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(dk, k_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(dv, v_host, tbytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return A2SF_ERR_CUDA;
+        rc = a2sf_prefill(p, n, dq, dk, dv, sb, sh, st, dout, dsc, dkept, nullptr, inner,
+                          prefill_ws_bytes(p, n), cuda_stream);
+        if (rc != A2SF_OK) return rc;
+        if (cudaMemcpyAsync(out_host, dout, tbytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaMemcpyAsync(scores_host, dsc, U * n * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+            cudaMemcpyAsync(kept_idx_host, dkept, U * m * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+            return A2SF_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return A2SF_ERR_CUDA;
+    } else {
+        cudaStream_t side[2] = {nullptr, nullptr};
+        cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
+        bool ok = cudaEventCreateWithFlags(&start, cudaEventDisableTiming) == cudaSuccess;
+        for (int x = 0; ok && x < 2; ++x)
+            ok = cudaStreamCreateWithFlags(&side[x], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&done[x], cudaEventDisableTiming) == cudaSuccess;
+        // work already queued on the caller's stream comes first
+        ok = ok && cudaEventRecord(start, s) == cudaSuccess;
+        for (int x = 0; ok && x < 2; ++x) ok = cudaStreamWaitEvent(side[x], start, 0) == cudaSuccess;
+        const size_t eb = elem_bytes(p->dtype);
+        const int rows_per = (p->B + chunks - 1) / chunks;
+        a2sf_params pc = *p;
+        pc.B = rows_per;
+        const size_t inner_half = align_up(prefill_ws_bytes(&pc, n));     // two of them fit: rows_per <= B/2 rounded up
+        const bool two_inner = 2 * inner_half <= prefill_ws_bytes(p, n);
+        int rc2 = A2SF_OK;
+        for (int c = 0; ok && rc2 == A2SF_OK && c * rows_per < p->B; ++c) {
+            const int b0 = c * rows_per, nb = (b0 + rows_per <= p->B) ? rows_per : p->B - b0;
+            // without room for two inner workspaces the chunks' kernels share one stream
+            cudaStream_t cs = side[two_inner ? (c & 1) : 0];
+            const size_t ub = (size_t)b0 * p->H, un = (size_t)nb * p->H;
+            const size_t off = ub * n * p->d * eb, len = un * n * p->d * eb;
+            ok = cudaMemcpyAsync((char *)dq + off, (const char *)q_host + off, len, cudaMemcpyHostToDevice, cs) == cudaSuccess &&
+                 cudaMemcpyAsync((char *)dk + off, (const char *)k_host + off, len, cudaMemcpyHostToDevice, cs) == cudaSuccess &&
+                 cudaMemcpyAsync((char *)dv + off, (const char *)v_host + off, len, cudaMemcpyHostToDevice, cs) == cudaSuccess;
+            if (!ok) break;
+            pc.B = nb;
+            rc2 = a2sf_prefill(&pc, n, (char *)dq + off, (char *)dk + off, (char *)dv + off, sb, sh, st,
+                               (char *)dout + off, dsc + ub * n, dkept + ub * m, nullptr,
+                               (char *)inner + ((two_inner && (c & 1)) ? inner_half : 0), inner_half, cs);
+            if (rc2 != A2SF_OK) break;
+            ok = cudaMemcpyAsync((char *)out_host + off, (char *)dout + off, len, cudaMemcpyDeviceToHost, cs) == cudaSuccess &&
+                 cudaMemcpyAsync(scores_host + ub * n, dsc + ub * n, un * n * 4, cudaMemcpyDeviceToHost, cs) == cudaSuccess &&
+                 cudaMemcpyAsync(kept_idx_host + ub * m, dkept + ub * m, un * m * 4, cudaMemcpyDeviceToHost, cs) == cudaSuccess;
+        }
+        // the caller's stream continues only after both side streams have drained
+        for (int x = 0; x < 2; ++x)
+            if (side[x] && done[x] && cudaEventRecord(done[x], side[x]) == cudaSuccess)
+                cudaStreamWaitEvent(s, done[x], 0);
+        const bool drained = cudaStreamSynchronize(s) == cudaSuccess;
+        for (int x = 0; x < 2; ++x) {
+            if (side[x]) { cudaStreamSynchronize(side[x]); cudaStreamDestroy(side[x]); }
+            if (done[x]) cudaEventDestroy(done[x]);
+        }
+        if (start) cudaEventDestroy(start);
+        if (rc2 != A2SF_OK) return rc2;
+        if (!ok || !drained) return A2SF_ERR_CUDA;
+    }
     if (dev_k) *dev_k = dk;
     if (dev_v) *dev_v = dv;
     if (dev_scores) *dev_scores = dsc;

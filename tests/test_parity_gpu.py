@@ -174,6 +174,27 @@ def test_host_buffer_entry_points_match_device_ones():
         assert torch.equal(a[key], b[key]), key
 
 
+@pytest.mark.parametrize("B", [2, 5, 9])
+def test_host_buffer_prefill_in_chunks_of_batch_rows_matches_the_device_call(B):
+    """With several batch rows the host-buffer prefill is pipelined over chunks of them on
+    internal streams; every result must still be the device call's, bit for bit."""
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W["opt_6p7b"].scaled(B=B, H=2, n=333)
+    q, k, v = wl.make_prompt(w)
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    out_d, S_d, kept_d, _ = a2sf.a2sf_prefill(p, q.cuda(), k.cuda(), v.cuda())
+    ws = torch.empty((a2sf.a2sf_prefill_host_workspace_bytes(p, w.n),), dtype=torch.uint8, device="cuda")
+    out_h = torch.empty_like(q).pin_memory()
+    S_h = torch.empty((w.B, w.H, w.n), dtype=torch.float32).pin_memory()
+    kept_h = torch.empty((w.B, w.H, w.budget), dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        out_h.zero_(); S_h.zero_(); kept_h.zero_()
+        a2sf.a2sf_prefill_host(p, w.n, q.pin_memory(), k.pin_memory(), v.pin_memory(), out_h, S_h, kept_h, ws)
+        assert torch.equal(out_h, out_d.cpu()) and torch.equal(S_h, S_d.cpu()) and torch.equal(kept_h, kept_d.cpu())
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+
+
 def test_export_import_round_trip_and_generator_on_device():
     from paper_2407_20485_b200 import binding as a2sf
 
