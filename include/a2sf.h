@@ -149,7 +149,10 @@ int a2sf_rescore_per_head(const a2sf_params *p, int32_t n,
  * asynchronous).  Inputs are copied to the device workspace, results copied back,
  * and the call returns after the stream has drained.  The device copies of k, v,
  * scores and kept_idx stay valid in the workspace for a2sf_cache_load: their
- * addresses are returned through dev_k, dev_v, dev_scores, dev_kept (any may be NULL). */
+ * addresses are returned through dev_k, dev_v, dev_scores, dev_kept (any may be NULL).
+ * With two or more batch rows the work is pipelined over chunks of rows on two streams that
+ * the call creates and destroys: they start after what is already queued on cuda_stream,
+ * and cuda_stream (and the call) continues only when they have drained. */
 size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n);
 
 int a2sf_prefill_host(const a2sf_params *p, int32_t n,
