@@ -257,7 +257,9 @@ def test_truncated_scoring_window_matches_partial_sum_and_respects_bound(name, k
                                           oracle.select(want[u], w.budget, w.recent))
         bound = a2sf.a2sf_score_window_bound(w.alpha, n, Wn)
         short = to_f64(S0).reshape(U, n) - got
-        assert short.min() >= -1e-4 * to_f64(S0).max() and short.max() <= bound * (1 + 1e-4) + 1e-30
+        # both score vectors carry fp32 rounding of their own, which dwarfs a tiny bound
+        slack = 4e-6 * to_f64(S0).max()
+        assert short.min() >= -1e-4 * to_f64(S0).max() and short.max() <= bound * (1 + 1e-4) + slack
         if Wn >= n:
             assert bound == 0.0 and torch.equal(S1, S0)
 
@@ -326,7 +328,7 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     q, k, v = wl.make_prompt(w, device="cuda")
     p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
     cache = a2sf.Cache(p)
-    q2 = q[:, :, 5:6].contiguous()
+    q2 = q[:, :, min(5, w.n - 1):min(5, w.n - 1) + 1].contiguous()
     cache.a2sf_decode_step(w.alpha, q2[:, :, 0], q2[:, :, 0], q2[:, :, 0],
                            torch.empty_like(q2[:, :, 0]),
                            torch.empty((w.B, w.H), dtype=torch.int32, device="cuda"))   # dirty the cache
@@ -616,3 +618,48 @@ def test_full_size_long_context_sweep():
     w = W["long_context"]
     units = _sample_units(w, 4 if EXHAUSTIVE else 2)
     _run(w, units=units, alphas=list(w.alphas), steps=w.steps if EXHAUSTIVE else 48, check_every=16)
+
+
+# ---- seeded random shapes and policies: a bounded sample of what a longer fuzzing run covers -------
+def _random_cases(seed, count):
+    import random
+
+    rng = random.Random(seed)
+    for _ in range(count):
+        M = rng.choice([1, 2, 3, 8, 17, 64, 100, 128, 205, 256, 512, 513])
+        yield dict(dtype=rng.choice(["fp32", "bf16", "fp16"]), d=rng.choice([64, 128]),
+                   B=rng.choice([1, 1, 2]), H=rng.choice([1, 2, 3]),
+                   n=rng.choice([1, 2, 7, 64, 127, 128, 129, 200, 255, 256, 257, 300, 513, 700]),
+                   budget=M, recent=rng.choice([0, 1, M // 2, max(M - 1, 0), M]),
+                   alpha=rng.choice([0.0, 0.1, 0.5, 0.9, 0.99, 1.0]))
+
+
+def test_random_shapes_and_policies_dense_prefill_and_decode():
+    import random
+
+    rng = random.Random(99)
+    for kw in _random_cases(20485, 40):
+        w = W["tiny_fp32"].scaled(steps=rng.choice([0, 1, 5, 20]), **kw)
+        _run(w, alphas=rng.choice([[], [0.0, 1.0], [0.7]]))
+
+
+def test_random_shapes_and_policies_widened_entry_points():
+    import contextlib
+    import io
+    import random
+
+    rng = random.Random(7)
+    for i, kw in enumerate(_random_cases(2407, 36)):
+        kw = dict(kw, n=min(kw["n"], 300))
+        with contextlib.redirect_stdout(io.StringIO()):
+            if i % 4 == 0:
+                test_streamed_prompt_against_the_oracle("tiny_fp32", kw)
+            elif i % 4 == 1:
+                G = rng.choice([1, 2, 3, 4, 8])
+                test_grouped_query_heads_against_the_oracle("tiny_fp32", dict(kw, steps=rng.choice([1, 7, 20])), G)
+            elif i % 4 == 2:
+                test_similarity_with_the_ideal_mask("tiny_fp32", kw)
+            else:
+                kw["alpha"] = kw["alpha"] or 0.5
+                test_truncated_scoring_window_matches_partial_sum_and_respects_bound(
+                    "tiny_fp32", kw, [1, rng.choice([2, 17, 64, 128, 130]), kw["n"], kw["n"] + 5])
