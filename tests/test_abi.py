@@ -135,3 +135,40 @@ def test_budget_beyond_the_documented_maximum_is_refused_on_the_host():
     assert a2sf.lib.a2sf_cache_bytes(ctypes.byref(ok)) > 0
     assert a2sf.lib.a2sf_cache_bytes(ctypes.byref(too_big)) == 0
     assert a2sf.lib.a2sf_prefill_workspace_bytes(ctypes.byref(too_big), 64) == 0
+
+
+def test_header_is_plain_c_and_links_from_a_c_program(tmp_path):
+    """include/a2sf.h compiled as strict C99 by gcc, linked against the library, and a few
+    host-only entry points called from C: no C++ or torch types at the boundary."""
+    import subprocess
+
+    from paper_2407_20485_b200 import binding
+
+    root = Path(__file__).resolve().parents[1]
+    src = tmp_path / "use_a2sf.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <string.h>
+#include "a2sf.h"
+int main(void)
+{
+    a2sf_params p;
+    memset(&p, 0, sizeof p);
+    p.B = 2; p.H = 4; p.d = 128; p.dtype = A2SF_BF16; p.budget = 64; p.recent = 32; p.alpha = 0.5f;
+    if (a2sf_cache_bytes(&p) == 0) return 1;
+    if (a2sf_prefill_workspace_bytes(&p, 300) == 0) return 2;
+    p.recent = 65;                                     /* recent > budget */
+    if (a2sf_cache_bytes(&p) != 0) return 3;
+    if (a2sf_decode_step(NULL, 0.5f, NULL, NULL, NULL, NULL, NULL, NULL) != A2SF_ERR_INVALID_ARG) return 4;
+    if (a2sf_score_window_bound(0.5f, 100, 3) <= 0.0) return 5;
+    printf("%s\n", a2sf_status_string(A2SF_ERR_WORKSPACE));
+    return 0;
+}
+''')
+    exe = tmp_path / "use_a2sf"
+    lib_dir = Path(binding._LIB_PATH).parent
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", str(root / "include"),
+                    str(src), "-o", str(exe), f"-L{lib_dir}", "-la2sf", f"-Wl,-rpath,{lib_dir}"], check=True)
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, (r.returncode, r.stdout, r.stderr)
+    assert len(r.stdout.strip()) > 0
