@@ -453,7 +453,10 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             // short units simply takes more of them.  The claim for the NEXT unit and its row
             // count are requested before the current unit is streamed, so neither round trip
             // ever stalls the copy stream.
-            int u_next = atomicAdd(&c.sched[0], 1);
+            // With no more units than CTAs the deal is static (unit = CTA index): the first
+            // claim's round trip to the counter would sit at the head of a very short kernel.
+            const bool static_deal = c.U <= (int)gridDim.x;
+            int u_next = static_deal ? (int)blockIdx.x : atomicAdd(&c.sched[0], 1);
             if (u_next >= c.U) u_next = -1;
             int cnt_next = u_next >= 0 ? min(c.count[u_next], M) : 0;
             for (uint32_t n_unit = 0; alive; ++n_unit) {
@@ -464,7 +467,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                 sh->cnt_q[qi] = cnt;
                 tc::mbar_arrive(&sh->uq_full[qi]);
                 if (u < 0) break;
-                u_next = atomicAdd(&c.sched[0], 1);
+                u_next = static_deal ? -1 : atomicAdd(&c.sched[0], 1);
                 if (u_next >= c.U) u_next = -1;
                 cnt_next = u_next >= 0 ? min(c.count[u_next], M) : 0;
                 for (int pass = 0; alive && pass < 2; ++pass) {
