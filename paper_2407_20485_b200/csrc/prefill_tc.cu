@@ -310,8 +310,11 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 //     S_A(0) S_B(0) | PV_A(0) S_A(1) | PV_B(0) S_B(1) | PV_A(1) S_A(2) | ...
 // so that while one stream's rows are in the softmax warps the other stream's MMAs run.
 //   S = Q K^T        -> TMEM, 128 fp32 columns per stream
-//   softmax warps    : two threads per row.  The running maximum is kept lazily (the accumulator
-//                      is rescaled only when the row maximum grows by more than 2^8).  P, rounded
+//   softmax warps    : two threads per row.  The row's reference (what is subtracted before the
+//                      exponential) moves lazily: a tile is first computed against the current
+//                      one and redone, with the exact row maximum and a rescaled accumulator,
+//                      only if its row sum shows that a probability may have left fp16's range.
+//                      P, rounded
 //                      to the storage type, is written back into the SAME tensor-memory columns
 //                      the logits came from and is read from there as the A operand of the next
 //                      MMA: shared-memory bandwidth is the scarce resource (two operands read
@@ -334,6 +337,7 @@ constexpr int kAttnThreads = 320;
 constexpr int kKStages = 3;                  // K tiles in flight
 constexpr int kVStages = 2;                  // V tiles in flight
 constexpr float kRescaleThreshold = 8.0f;    // log2 units
+constexpr float kOptimisticLimit = 32768.f;  // a row sum below this keeps every probability < 2^15
 
 struct AttnArgs {
     void *out;            // [B][H][n][d], strides below
@@ -588,66 +592,86 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
                     for (int x = 0; x < 32; ++x)
                         if (half * 64 + c * 32 + x > r) v[c][x] = 0xff800000u;
             }
-            // pass 1: row maximum; the two threads of a row exchange theirs through shared memory
-            float mx[2];
+            // Probabilities against the reference -neg_m, packed in pairs over the thread's own
+            // logits columns (which are in registers by now); returns their sum.
+            auto write_p = [&](float neg_m) -> float {
+                float rs[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                mx[c] = max3(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]), __uint_as_float(v[c][2]));
-#pragma unroll
-                for (int x = 3; x + 1 < 32; x += 2)
-                    mx[c] = max3(mx[c], __uint_as_float(v[c][x]), __uint_as_float(v[c][x + 1]));
-                mx[c] = fmaxf(mx[c], __uint_as_float(v[c][31]));
-            }
-            const float own = fmaxf(mx[0], mx[1]);
-            sh->xch[X][half][r] = own;
-            named_barrier(1 + quarter, 64);                // this quarter's two warps
-            const float smax = fmaxf(own, sh->xch[X][half ^ 1][r]);
-            // Lazy maximum (log2 domain): the reference moves only on the first tile or when
-            // the row maximum exceeds it by more than 2^8; otherwise probabilities up to 256
-            // are simply kept.  Both threads of a row see the same smax and decide alike.
-            const float xmax = fmaf(smax, a.sl2, -m_used[X]);
-            const bool grow = (t == 0) || (xmax > kRescaleThreshold);
-            float factor = 1.f;
-            if (grow) {
-                m_used[X] += xmax;
-                factor = t == 0 ? 0.f : ex2_approx(-xmax);
-            }
-            if (t > 0 && __any_sync(0xffffffffu, grow)) {
-                // O_X holds tiles 0..t-1 once the previous P V product has retired
-                wait(&sh->o_done[X], (t - 1) & 1);
-                tc_fence_after_sync();
-#pragma unroll 1
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(to + c * 32, o);
-                    tmem_wait_ld();
+                    uint32_t hi[16], lo[16];
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * factor);
-                    tmem_st32(to + c * 32, o);
+                    for (int e = 0; e < 16; ++e) {
+                        const float p0 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e]), a.sl2, neg_m));
+                        const float p1 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e + 1]), a.sl2, neg_m));
+                        rs[e & 3] += p0 + p1;
+                        hi[e] = pack2<PT>(p0, p1);
+                        if (kSplitP)      // a bf16 is the upper half of an fp32
+                            lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
+                                             p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    }
+                    tmem_st16(sp + c * 16, hi);
+                    if (kSplitP) tmem_st16(sp + 32 + c * 16, lo);
                 }
-                tmem_wait_st();
+                return (rs[0] + rs[1]) + (rs[2] + rs[3]);
+            };
+            // Optimistic tile: keep the row's reference and look at the result.  The sum bounds
+            // every probability, so a sum within kOptimisticLimit means that none has left
+            // fp16's range; the row maximum is then never computed.  Both threads of a row (and
+            // both warps of the quarter) take the same decision.
+            float factor = 1.f, rowsum = 0.f;
+            bool exact = (t == 0);
+            if (!exact) {
+                rowsum = write_p(-m_used[X]);
+                const bool bad = !(rowsum <= kOptimisticLimit);          // also NaN
+                sh->xch[X][half][r] = bad ? 1.f : 0.f;
+                named_barrier(1 + quarter, 64);                // this quarter's two warps
+                const bool pair_bad = bad || sh->xch[X][half ^ 1][r] != 0.f;
+                exact = __any_sync(0xffffffffu, pair_bad);
+                if (exact) named_barrier(1 + quarter, 64);     // flags read before the buffer is reused
             }
-            // pass 2: probabilities, packed in pairs over the thread's own logits columns
-            const float neg_m = -m_used[X];
-            float rs[4] = {0.f, 0.f, 0.f, 0.f};
+            if (exact) {
+                // row maximum; the two threads of a row exchange theirs through shared memory
+                float mx[2];
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t hi[16], lo[16];
+                for (int c = 0; c < 2; ++c) {
+                    mx[c] = max3(__uint_as_float(v[c][0]), __uint_as_float(v[c][1]), __uint_as_float(v[c][2]));
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e]), a.sl2, neg_m));
-                    const float p1 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e + 1]), a.sl2, neg_m));
-                    rs[e & 3] += p0 + p1;
-                    hi[e] = pack2<PT>(p0, p1);
-                    if (kSplitP)      // a bf16 is the upper half of an fp32
-                        lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
-                                         p1 - __uint_as_float(hi[e] & 0xffff0000u));
+                    for (int x = 3; x + 1 < 32; x += 2)
+                        mx[c] = max3(mx[c], __uint_as_float(v[c][x]), __uint_as_float(v[c][x + 1]));
+                    mx[c] = fmaxf(mx[c], __uint_as_float(v[c][31]));
                 }
-                tmem_st16(sp + c * 16, hi);
-                if (kSplitP) tmem_st16(sp + 32 + c * 16, lo);
+                const float own = fmaxf(mx[0], mx[1]);
+                sh->xch[X][half][r] = own;
+                named_barrier(1 + quarter, 64);
+                const float smax = fmaxf(own, sh->xch[X][half ^ 1][r]);
+                // The reference moves only on the first tile or when the row maximum exceeds it
+                // by more than 2^8 (log2 domain); a row that overflowed the optimistic limit is
+                // at least 2^9 above it.
+                const float xmax = fmaf(smax, a.sl2, -m_used[X]);
+                const bool grow = (t == 0) || (xmax > kRescaleThreshold);
+                if (grow) {
+                    m_used[X] += xmax;
+                    factor = t == 0 ? 0.f : ex2_approx(-xmax);
+                }
+                if (t > 0 && __any_sync(0xffffffffu, grow)) {
+                    // O_X holds tiles 0..t-1 once the previous P V product has retired
+                    wait(&sh->o_done[X], (t - 1) & 1);
+                    tc_fence_after_sync();
+#pragma unroll 1
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(to + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int x = 0; x < 32; ++x) o[x] = __float_as_uint(__uint_as_float(o[x]) * factor);
+                        tmem_st32(to + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+                rowsum = write_p(-m_used[X]);
             }
             tmem_wait_st();
-            l[X] = fmaf(l[X], factor, (rs[0] + rs[1]) + (rs[2] + rs[3]));
+            l[X] = fmaf(l[X], factor, rowsum);
             tc_fence_before_sync();
             mbar_arrive(&sh->p_full[X]);
         };

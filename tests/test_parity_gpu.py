@@ -132,6 +132,36 @@ def test_values_beyond_fp16_range_take_the_bf16_product():
         np.testing.assert_array_equal(kept.cpu().numpy()[0], ref["kept"])
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+def test_late_dominant_keys_force_the_softmax_reference_to_move(dtype):
+    """The attention pass keeps a row's softmax reference while the tile's probabilities stay in
+    range and recomputes the tile when they do not: keys whose logits dwarf everything before
+    them, placed in late tiles, must take that path and still match the oracle."""
+    import oracle
+    from parity_util import ParityReport, check_out, check_scores, to_f64
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W["llama2_7b"].scaled(H=3, n=900, dtype=dtype)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    k = k.clone()
+    for pos, gain in ((300, 6.0), (301, 9.0), (555, 14.0), (800, 25.0)):       # each beyond the last by 2^10 and more
+        k[:, :, pos] = (q[:, :, pos].float() * gain / 8.0).to(k.dtype)          # aligned with the later queries' typical direction
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    out, S, kept, lse = a2sf.a2sf_prefill(p, q, k, v)
+    torch.cuda.synchronize()
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+    U, n = w.units, w.n
+    Q, K, V = (to_f64(t).reshape(U, n, w.d) for t in (q, k, v))
+    ref = oracle.prefill(Q, K, V, w.scale, [w.alpha], w.budget, w.recent, nthreads=oracle.host_threads())
+    rep = ParityReport()
+    assert np.isfinite(to_f64(out)).all()
+    check_out(to_f64(out).reshape(U, n, w.d), ref["out"], w.dtype, rep, "out")
+    assert np.abs(to_f64(lse).reshape(U, n) - ref["lse"]).max() <= 1e-4 * max(1.0, np.abs(ref["lse"]).max())
+    check_scores(to_f64(S).reshape(U, n), ref["S"][:, 0], rep, "scores")
+    # the planted rows really do dominate: their own logit is far above the earlier maximum
+    assert (ref["lse"][:, 800] - ref["lse"][:, 799]).min() > 20.0
+
+
 def test_host_buffer_entry_points_match_device_ones():
     from paper_2407_20485_b200 import binding as a2sf
 
