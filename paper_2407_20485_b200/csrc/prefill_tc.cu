@@ -326,12 +326,14 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
 // Warp roles (320 threads): warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2-9
 // softmax + epilogue: two threads per query row (64 logits each), all eight warps on one
 // stream's tile at a time, the streams taken in turn.
-// Measured on the longest CTA (63 stream tiles, 2393 clocks each against 1440 of tensor work):
-// the softmax warps spend 65 % of their time in the exponential pass at ~12 clocks per logit
-// per scheduler -- the special-function unit issues one warp instruction per 8 clocks and the
-// other ~3.5 instructions per logit do not hide behind it.  Moving part of the exponentials to
-// an FMA-pipe polynomial (+11 instructions each) or the fp16 packing to integer instructions
-// made the pass slower, so neither is used.
+// Measured on the longest CTA (63 stream tiles, 2393 clocks each against 1440 of tensor work,
+// before the row-maximum pass became the exception): the softmax warps spent 65 % of their time
+// in the exponential pass at ~12 clocks per logit per scheduler -- the special-function unit
+// issues one warp instruction per 8 clocks and the other ~3.5 instructions per logit do not hide
+// behind it -- and 8 % on the row maximum.  Every instruction per logit counts: dropping the
+// maximum pass from the common path paid, while moving part of the exponentials to an FMA-pipe
+// polynomial (+11 instructions each) or the fp16 packing to integer instructions made the
+// pass slower, so neither is used.
 // ============================================================================================
 constexpr int kAttnThreads = 320;
 constexpr int kKStages = 3;                  // K tiles in flight
