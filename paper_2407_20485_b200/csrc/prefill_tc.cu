@@ -69,6 +69,29 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+// Two fp32 operations per instruction (sm_100 packed arithmetic on register pairs).
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float y;
@@ -597,15 +620,19 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
             // Probabilities against the reference -neg_m, packed in pairs over the thread's own
             // logits columns (which are in registers by now); returns their sum.
             auto write_p = [&](float neg_m) -> float {
-                float rs[4] = {0.f, 0.f, 0.f, 0.f};
+                // multiply-add and row sum on register pairs: one instruction per two logits
+                const uint64_t sl2x2 = pack_f32x2(__float_as_uint(a.sl2), __float_as_uint(a.sl2));
+                const uint64_t nmx2 = pack_f32x2(__float_as_uint(neg_m), __float_as_uint(neg_m));
+                uint64_t rs2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t hi[16], lo[16];
 #pragma unroll
                     for (int e = 0; e < 16; ++e) {
-                        const float p0 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e]), a.sl2, neg_m));
-                        const float p1 = ex2_approx(fmaf(__uint_as_float(v[c][2 * e + 1]), a.sl2, neg_m));
-                        rs[e & 3] += p0 + p1;
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(v[c][2 * e], v[c][2 * e + 1]), sl2x2, nmx2), x0, x1);
+                        const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                        rs2[e & 3] = add_f32x2(rs2[e & 3], pack_f32x2(__float_as_uint(p0), __float_as_uint(p1)));
                         hi[e] = pack2<PT>(p0, p1);
                         if (kSplitP)      // a bf16 is the upper half of an fp32
                             lo[e] = pack2<PT>(p0 - __uint_as_float(hi[e] << 16),
@@ -614,7 +641,10 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
                     tmem_st16(sp + c * 16, hi);
                     if (kSplitP) tmem_st16(sp + 32 + c * 16, lo);
                 }
-                return (rs[0] + rs[1]) + (rs[2] + rs[3]);
+                float rs[8];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) unpack_f32x2(rs2[x], rs[2 * x], rs[2 * x + 1]);
+                return ((rs[0] + rs[1]) + (rs[2] + rs[3])) + ((rs[4] + rs[5]) + (rs[6] + rs[7]));
             };
             // Optimistic tile: keep the row's reference and look at the result.  The sum bounds
             // every probability, so a sum within kOptimisticLimit means that none has left
