@@ -191,6 +191,19 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         for (int x = 0; x < kScoreCRing; ++x) mbar_init(&sh->c_ready[x], 1);
         sh->abort_flag = 0;
         fence_mbar_init();
+        // the K block and the first query tiles are requested here, before the tensor-memory
+        // allocation and the CTA-wide barrier, so that their latency overlaps the set-up
+        prefetch_tmap(&tmap_q);
+        prefetch_tmap(&tmap_k);
+        mbar_arrive_expect_tx(&sh->k_full, kTileBytes);
+        tma_load_4d(Ks, &tmap_k, &sh->k_full, 0, kb * kBlk, h / a.G, b);
+        tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full, 64, kb * kBlk, h / a.G, b);
+        for (int it = 0; it < kScoreStages && it < ntiles; ++it) {
+            mbar_arrive_expect_tx(&sh->q_full[it], kTileBytes);
+            uint8_t *dst = Qs + it * kTileBytes;
+            tma_load_4d(dst, &tmap_q, &sh->q_full[it], 0, (t_first + it) * kBlk, h, b);
+            tma_load_4d(dst + kHalfBytes, &tmap_q, &sh->q_full[it], 64, (t_first + it) * kBlk, h, b);
+        }
     }
     if (warp == 1) {
         tmem_alloc(&sh->tmem_base, 256);
@@ -207,14 +220,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         // They are written one tile ahead of the tensor core, so the epilogue warps never meet
         // at a barrier of their own and drift freely against each other.
         const float *lse = a.lse + (size_t)u * a.n;
-        if (lane == 0) {
-            prefetch_tmap(&tmap_q);
-            prefetch_tmap(&tmap_k);
-            mbar_arrive_expect_tx(&sh->k_full, kTileBytes);
-            tma_load_4d(Ks, &tmap_k, &sh->k_full, 0, kb * kBlk, h / a.G, b);
-            tma_load_4d(Ks + kHalfBytes, &tmap_k, &sh->k_full, 64, kb * kBlk, h / a.G, b);
-        }
-        int issued = 0;
+        int issued = min(ntiles, kScoreStages);      // requested during set-up
         for (int it = 0; it < ntiles; ++it) {
             const int s = it % kScoreStages;
             const uint32_t ph = (it / kScoreStages) & 1;
@@ -229,7 +235,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
                                 : INFINITY;
             }
             int ok = 1;
-            if (lane == 0) {
+            if (lane == 0 && it >= kScoreStages) {
                 ok = mbar_wait(&sh->q_empty[s], ph ^ 1, abort_flag) ? 1 : 0;
                 if (ok) {
                     mbar_arrive_expect_tx(&sh->q_full[s], kTileBytes);
@@ -240,7 +246,7 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
-            issued = it + 1;
+            issued = max(issued, it + 1);
             *reinterpret_cast<float4 *>(&sh->cbuf[it % kScoreCRing][lane * 4]) =
                 make_float4(c4[0], c4[1], c4[2], c4[3]);
             __syncwarp();
