@@ -36,7 +36,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode_step_stream_kernel launch (ncu, config 4;
 # the capture is summarised in profiles/launch_list_llama2_13b.md).  Set to None when the kernel changes.
-NCU_DECODE_TRAFFIC = {("llama2_13b", 32): 343290000}
+NCU_DECODE_TRAFFIC = {("llama2_13b", 32): 342910000}
 
 
 def load_peaks():
