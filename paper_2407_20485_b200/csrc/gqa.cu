@@ -30,7 +30,10 @@ __global__ void group_sum_kernel(const float *__restrict__ per_head, float *__re
     }
 }
 
-template <typename T, int D>
+// GMAX: compile-time bound of the group size (2, 4 or 8): the per-lane query slices and
+// accumulator rows are sized by it, and smaller groups leave room for more CTAs per SM, i.e. more
+// loads in flight (the kernel is bound by load latency).
+template <typename T, int D, int GMAX>
 __global__ void __launch_bounds__(kGroupThreads)
 decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ q,
                          const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ out,
@@ -63,14 +66,14 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     const T *knu = k_new + (size_t)u * D, *vnu = v_new + (size_t)u * D;
 
     // this lane's slice of every query
-    float qf[kMaxGroup][VEC];
+    float qf[GMAX][VEC];
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g)
+    for (int g = 0; g < GMAX; ++g)
         if (g < G) Elem<T>::unpack(*reinterpret_cast<const uint4 *>(qu + (size_t)g * D + sub * VEC), qf[g]);
 
     // ---- (i) logits of the cached keys and of the new key, for every query of the group -----
     // kUnroll row groups per iteration, their loads issued before any arithmetic
-    constexpr int kUnroll = 4;
+    constexpr int kUnroll = GMAX <= 4 ? 8 : 4;
     for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
         uint4 raw[kUnroll];
 #pragma unroll
@@ -86,7 +89,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
             float kf[VEC];
             Elem<T>::unpack(raw[x], kf);
 #pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
+            for (int g = 0; g < GMAX; ++g) {
                 if (g < G) {
                     float dot = 0.f;
 #pragma unroll
@@ -119,9 +122,9 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     __syncthreads();
 
     // ---- (iii) out_g = sum_slot a_g[slot] V[slot] + a_g[self] v_new -----------------------------
-    float acc[kMaxGroup][VEC];
+    float acc[GMAX][VEC];
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g)
+    for (int g = 0; g < GMAX; ++g)
 #pragma unroll
         for (int e = 0; e < VEC; ++e) acc[g][e] = 0.f;
     for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
@@ -140,7 +143,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
                 float vf[VEC];
                 Elem<T>::unpack(raw[x], vf);
 #pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) {
+                for (int g = 0; g < GMAX; ++g) {
                     if (g < G) {
                         const float a = w[g * wstride + s];
 #pragma unroll
@@ -151,7 +154,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
         }
     }
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) {
+    for (int g = 0; g < GMAX; ++g) {
         if (g < G) {
 #pragma unroll
             for (int e = 0; e < VEC; ++e) {
@@ -230,14 +233,14 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     }
 }
 
-template <typename T, int D>
-cudaError_t launch_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
-                         const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+template <typename T, int D, int GMAX>
+cudaError_t launch_group_n(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                           const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
     const size_t wstride = ((size_t)c.M + 1 + 3) & ~(size_t)3;
     const size_t smem = ((size_t)G * wstride + (size_t)(kGroupThreads / 32) * G * D) * sizeof(float);
     if (smem > 220 * 1024) return cudaErrorInvalidValue;
-    auto kern = decode_step_group_kernel<T, D>;
+    auto kern = decode_step_group_kernel<T, D, GMAX>;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -246,6 +249,15 @@ cudaError_t launch_group(const CacheView &c, int G, float alpha, const void *q, 
                                            static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
     count_launch();
     return cudaGetLastError();
+}
+
+template <typename T, int D>
+cudaError_t launch_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                         const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    if (G <= 2) return launch_group_n<T, D, 2>(c, G, alpha, q, k_new, v_new, out, evicted, s);
+    if (G <= 4) return launch_group_n<T, D, 4>(c, G, alpha, q, k_new, v_new, out, evicted, s);
+    return launch_group_n<T, D, 8>(c, G, alpha, q, k_new, v_new, out, evicted, s);
 }
 
 }  // namespace
