@@ -550,6 +550,40 @@ def test_several_tokens_in_one_call_equal_single_steps():
         assert torch.equal(s1[key], s2[key]), key
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("llama2_7b", dict(H=3, n=700)),            # bf16 tensor-core passes (V conversion, flag, one attention launch)
+    ("tiny_fp32", dict(n=300, budget=64, recent=32)),
+])
+def test_prefill_and_cache_load_replayed_from_a_cuda_graph(name, kw):
+    from paper_2407_20485_b200 import binding as a2sf
+
+    w = W[name].scaled(**kw)
+    q, k, v = wl.make_prompt(w, device="cuda")
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    out0, S0, kept0, lse0 = a2sf.a2sf_prefill(p, q, k, v)                 # direct call (also the warm-up)
+    ref = a2sf.Cache(p)
+    ref.a2sf_cache_load(k, v, S0, kept0)
+    out, S, kept, lse = (torch.zeros_like(t) for t in (out0, S0, kept0, lse0))
+    ws = torch.empty((max(256, a2sf.a2sf_prefill_workspace_bytes(p, w.n)),), dtype=torch.uint8, device="cuda")
+    cache = a2sf.Cache(p)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        a2sf.a2sf_prefill(p, q, k, v, out=out, scores=S, kept_idx=kept, lse=lse, workspace=ws)
+        cache.a2sf_cache_load(k, v, S, kept)
+    for _ in range(2):
+        for t in (out, S, kept, lse):
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, out0) and torch.equal(S, S0) and torch.equal(kept, kept0) and torch.equal(lse, lse0)
+        a_, b_ = ref.a2sf_cache_export(), cache.a2sf_cache_export()
+        torch.cuda.synchronize()
+        for key in a_:
+            assert torch.equal(a_[key], b_[key]), key
+    assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+
+
 def test_graphed_steps_helper_continues_a_cache_like_single_calls():
     from paper_2407_20485_b200 import binding as a2sf
     from paper_2407_20485_b200.graphs import GraphedSteps
