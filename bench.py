@@ -351,7 +351,8 @@ def run_ours(args):
         # stepped as a rotation over the named model's layer count (not part of the headline)
         result["decode_layer_rotation"] = [
             decode_layer_rotation(a2sf, dev, name, layers, args.rotation_steps, args.rotation_reps)
-            for name, layers in (("llama2_7b", 32), ("opt_6p7b", 32), ("long_context", 32))]
+            for name, layers in (("llama2_7b", 32), ("opt_6p7b", 32), ("long_context", 32),
+                                 ("llama2_13b", 1))]          # the headline workload, graph-replayed
     if rank == 0:
         print(json.dumps(result))
     a2dist.finalize()
@@ -374,7 +375,7 @@ def decode_layer_rotation(a2sf, dev, name, layers, steps, reps):
                        f"budget{w.budget} recent{w.recent}",
            "bytes_per_launch": bytes_per_launch, "steps_per_replay": steps, "repetitions": reps,
            "timing": "one CUDA-graph replay of steps x layers launches between two events"}
-    for L in (1, layers):
+    for L in sorted({1, layers}):
         caches = [a2sf.Cache(p, dev) for _ in range(L)]
         o = torch.empty((L, w.B, w.H, w.d), dtype=w.torch_dtype, device=dev)
         e = torch.empty((L, w.B, w.H), dtype=torch.int32, device=dev)
