@@ -30,11 +30,53 @@ __global__ void group_sum_kernel(const float *__restrict__ per_head, float *__re
     }
 }
 
+// floats of shared memory per kernel instance, shared with the host-side size check
+__host__ __device__ inline size_t group_wstride(int M) { return ((size_t)M + 1 + 3) & ~(size_t)3; }
+
+__device__ __forceinline__ void cp_async4(void *smem_dst, const void *gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+                 "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// GMAX dot products, each spread over the LPR lanes of a row, are summed with a halving
+// butterfly: at every step a lane passes on the half of its values that its partner keeps, so
+// the whole reduction takes GMAX - 1 + log2(LPR / GMAX) shuffles instead of GMAX * log2(LPR).
+// Afterwards every lane holds the total of query  sub / (LPR / GMAX).
+template <int GMAX, int LPR>
+__device__ __forceinline__ float group_reduce(float (&d)[GMAX], int sub)
+{
+    static_assert(GMAX <= LPR, "one lane per query at least");
+    int nv = GMAX;
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) {
+        if (nv > 1) {
+            nv >>= 1;
+            const bool upper = (sub & o) != 0;
+#pragma unroll
+            for (int i = 0; i < GMAX / 2; ++i) {
+                if (i < nv) {
+                    const float send = upper ? d[i] : d[i + nv];
+                    const float keep = upper ? d[i + nv] : d[i];
+                    d[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                }
+            }
+        } else {
+            d[0] += __shfl_xor_sync(0xffffffffu, d[0], o);
+        }
+    }
+    return d[0];
+}
+
 // GMAX: compile-time bound of the group size (2, 4 or 8): the per-lane query slices and
-// accumulator rows are sized by it, and smaller groups leave room for more CTAs per SM, i.e. more
-// loads in flight (the kernel is bound by load latency).
+// accumulator rows are sized by it.  One CTA per K/V unit.  The kernel is a chain of dependent
+// phases around little data, so every global word it needs is requested as early as it can be:
+// the unit's scores and positions go to shared memory asynchronously at the start, K and V rows
+// are loaded one batch of kUnroll row groups ahead of the arithmetic, and the first V batch is
+// requested before the softmax.
 template <typename T, int D, int GMAX>
-__global__ void __launch_bounds__(kGroupThreads)
+__global__ void __launch_bounds__(kGroupThreads, 2)
 decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ q,
                          const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ out,
                          int32_t *__restrict__ evicted)
@@ -43,12 +85,16 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     constexpr int LPR = D / VEC;              // lanes per row
     constexpr int RPW = 32 / LPR;             // rows per warp-wide load
     constexpr int NW = kGroupThreads / 32;
+    constexpr int LPG = LPR / GMAX;           // lanes that end up with the same query's logit
     const int M = c.M;
-    const int wstride = (M + 1 + 3) & ~3;     // floats per query head in w[]
+    const int wstride = (int)group_wstride(M);
 
     extern __shared__ __align__(16) float gsm[];
     float *w = gsm;                                   // [G][wstride] logits, then probabilities
     float *part = w + (size_t)G * wstride;            // [NW][G][D] partial outputs
+    float *s_old = part + (size_t)NW * G * D;         // [wstride] the unit's scores before the step
+    int32_t *s_pos = reinterpret_cast<int32_t *>(s_old + wstride);   // [wstride] positions
+    __shared__ float red_m[NW][GMAX], red_l[NW][GMAX];
     __shared__ unsigned long long red_key[NW];
     __shared__ int red_slot[NW];
     __shared__ int s_target;
@@ -65,60 +111,100 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     const T *qu = q + (size_t)u * G * D;              // [G][D]
     const T *knu = k_new + (size_t)u * D, *vnu = v_new + (size_t)u * D;
 
-    // this lane's slice of every query
+    // scores and positions: thread tid stages, and later reads, slots tid, tid + 256, ...
+    for (int s = tid; s < cnt; s += kGroupThreads) {
+        cp_async4(s_old + s, Su + s);
+        cp_async4(s_pos + s, posu + s);
+    }
+
+    // this lane's slice of every query (zero for the unused heads of the bound)
     float qf[GMAX][VEC];
 #pragma unroll
-    for (int g = 0; g < GMAX; ++g)
-        if (g < G) Elem<T>::unpack(*reinterpret_cast<const uint4 *>(qu + (size_t)g * D + sub * VEC), qf[g]);
+    for (int g = 0; g < GMAX; ++g) {
+        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+        if (g < G) raw = *reinterpret_cast<const uint4 *>(qu + (size_t)g * D + sub * VEC);
+        Elem<T>::unpack(raw, qf[g]);
+    }
 
-    // ---- (i) logits of the cached keys and of the new key, for every query of the group -----
-    // kUnroll row groups per iteration, their loads issued before any arithmetic
     constexpr int kUnroll = GMAX <= 4 ? 8 : 4;
-    for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
-        uint4 raw[kUnroll];
+    constexpr int kBatch = NW * RPW * kUnroll;        // rows per batch of the whole CTA
+    // rows 0..cnt-1 are cached, row cnt is the new token's
+    auto load_rows = [&](uint4(&raw)[kUnroll], int s0, const T *base, const T *fresh) {
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
             const int s = s0 + x * NW * RPW + rsel;
             raw[x] = make_uint4(0u, 0u, 0u, 0u);
             if (s <= cnt)
-                raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? Ku + (size_t)s * D : knu) + sub * VEC);
+                raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? base + (size_t)s * D : fresh) + sub * VEC);
         }
+    };
+
+    // ---- (i) logits of the cached keys and of the new key, for every query of the group -----
+    uint4 cur[kUnroll], nxt[kUnroll];
+    load_rows(cur, warp * RPW, Ku, knu);
+    for (int s0 = warp * RPW; s0 <= cnt; s0 += kBatch) {
+        load_rows(nxt, s0 + kBatch, Ku, knu);         // nothing is loaded past row cnt
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
             const int s = s0 + x * NW * RPW + rsel;
             float kf[VEC];
-            Elem<T>::unpack(raw[x], kf);
+            Elem<T>::unpack(cur[x], kf);
+            float dot[GMAX];
 #pragma unroll
             for (int g = 0; g < GMAX; ++g) {
-                if (g < G) {
-                    float dot = 0.f;
+                dot[g] = 0.f;
 #pragma unroll
-                    for (int e = 0; e < VEC; ++e) dot = fmaf(qf[g][e], kf[e], dot);
-#pragma unroll
-                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    if (sub == 0 && s <= cnt) w[g * wstride + s] = dot * c.scale;
-                }
+                for (int e = 0; e < VEC; ++e) dot[g] = fmaf(qf[g][e], kf[e], dot[g]);
             }
+            const float tot = group_reduce<GMAX, LPR>(dot, sub);
+            const int g = sub / LPG;
+            if (sub % LPG == 0 && g < G && s <= cnt) w[g * wstride + s] = tot * c.scale;
         }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) cur[x] = nxt[x];
     }
+    // the first values are on their way while the softmax runs
+    load_rows(cur, warp * RPW, Vu, vnu);
     __syncthreads();
 
-    // ---- (ii) one softmax per query: warp g owns query g ---------------------------------------
-    for (int g = warp; g < G; g += NW) {
-        float *wg = w + g * wstride;
+    // ---- (ii) one softmax per query, all threads on every query ----------------------------------
+    float mg[GMAX], inv[GMAX];
+#pragma unroll
+    for (int g = 0; g < GMAX; ++g) {
         float m = -INFINITY;
-        for (int s = lane; s <= cnt; s += 32) m = fmaxf(m, wg[s]);
+        if (g < G)
+            for (int s = tid; s <= cnt; s += kGroupThreads) m = fmaxf(m, w[g * wstride + s]);
         m = warp_max(m);
-        float l = 0.f;
-        for (int s = lane; s <= cnt; s += 32) {
-            const float e = expf(wg[s] - m);
-            wg[s] = e;
-            l += e;
-        }
-        l = warp_sum(l);
-        const float inv = 1.f / l;
-        for (int s = lane; s <= cnt; s += 32) wg[s] *= inv;       // probabilities from here on
+        if (lane == 0) red_m[warp][g] = m;
     }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < GMAX; ++g) {
+        float m = red_m[0][g];
+#pragma unroll
+        for (int x = 1; x < NW; ++x) m = fmaxf(m, red_m[x][g]);
+        mg[g] = m;
+        float l = 0.f;
+        if (g < G)
+            for (int s = tid; s <= cnt; s += kGroupThreads) {
+                const float e = expf(w[g * wstride + s] - m);
+                w[g * wstride + s] = e;
+                l += e;
+            }
+        l = warp_sum(l);
+        if (lane == 0) red_l[warp][g] = l;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < GMAX; ++g) {
+        float l = red_l[0][g];
+#pragma unroll
+        for (int x = 1; x < NW; ++x) l += red_l[x][g];                  // fixed order
+        inv[g] = 1.f / l;
+        if (g < G)
+            for (int s = tid; s <= cnt; s += kGroupThreads) w[g * wstride + s] *= inv[g];   // probabilities
+    }
+    (void)mg;
     __syncthreads();
 
     // ---- (iii) out_g = sum_slot a_g[slot] V[slot] + a_g[self] v_new -----------------------------
@@ -127,21 +213,14 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     for (int g = 0; g < GMAX; ++g)
 #pragma unroll
         for (int e = 0; e < VEC; ++e) acc[g][e] = 0.f;
-    for (int s0 = warp * RPW; s0 <= cnt; s0 += NW * RPW * kUnroll) {
-        uint4 raw[kUnroll];
-#pragma unroll
-        for (int x = 0; x < kUnroll; ++x) {
-            const int s = s0 + x * NW * RPW + rsel;
-            raw[x] = make_uint4(0u, 0u, 0u, 0u);
-            if (s <= cnt)
-                raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? Vu + (size_t)s * D : vnu) + sub * VEC);
-        }
+    for (int s0 = warp * RPW; s0 <= cnt; s0 += kBatch) {
+        load_rows(nxt, s0 + kBatch, Vu, vnu);
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) {
             const int s = s0 + x * NW * RPW + rsel;
             if (s <= cnt) {
                 float vf[VEC];
-                Elem<T>::unpack(raw[x], vf);
+                Elem<T>::unpack(cur[x], vf);
 #pragma unroll
                 for (int g = 0; g < GMAX; ++g) {
                     if (g < G) {
@@ -152,6 +231,8 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
                 }
             }
         }
+#pragma unroll
+        for (int x = 0; x < kUnroll; ++x) cur[x] = nxt[x];
     }
 #pragma unroll
     for (int g = 0; g < GMAX; ++g) {
@@ -165,6 +246,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
             }
         }
     }
+    cp_async_wait_all();                       // this thread's staged scores and positions
     __syncthreads();
     for (int x = tid; x < G * D; x += kGroupThreads) {
         float o = 0.f;
@@ -181,9 +263,9 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     for (int s = tid; s < cnt; s += kGroupThreads) {
         float gain = 0.f;
         for (int g = 0; g < G; ++g) gain += w[g * wstride + s];
-        const float sn = fmaf(alpha, Su[s], gain);
+        const float sn = fmaf(alpha, s_old[s], gain);
         Su[s] = sn;
-        const int ps = posu[s];
+        const int ps = s_pos[s];
         if (full && ps <= newest_evictable) {
             const unsigned long long key = ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
             if (key < best) { best = key; best_slot = s; }
@@ -237,8 +319,7 @@ template <typename T, int D, int GMAX>
 cudaError_t launch_group_n(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
                            const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
-    const size_t wstride = ((size_t)c.M + 1 + 3) & ~(size_t)3;
-    const size_t smem = ((size_t)G * wstride + (size_t)(kGroupThreads / 32) * G * D) * sizeof(float);
+    const size_t smem = decode_group_smem_bytes(c.M, G, D);
     if (smem > 220 * 1024) return cudaErrorInvalidValue;
     auto kern = decode_step_group_kernel<T, D, GMAX>;
     if (smem > 48 * 1024) {
@@ -273,8 +354,8 @@ cudaError_t launch_group_sum(const float *per_head, float *out, int G, int n, si
 
 size_t decode_group_smem_bytes(int M, int G, int d)
 {
-    const size_t wstride = ((size_t)M + 1 + 3) & ~(size_t)3;
-    return ((size_t)G * wstride + (size_t)(kGroupThreads / 32) * G * d) * sizeof(float);
+    // logits [G][wstride], partial outputs [warps][G][d], staged scores and positions [wstride] each
+    return ((size_t)(G + 2) * group_wstride(M) + (size_t)(kGroupThreads / 32) * G * d) * sizeof(float);
 }
 
 cudaError_t launch_decode_step_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
