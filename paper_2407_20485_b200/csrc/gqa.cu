@@ -315,6 +315,343 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     }
 }
 
+// ---- 16-bit storage: the group's products on the tensor cores -----------------------------------
+// With G queries per K/V row the step is a skinny matrix product, [slots x d] . [d x G]: the
+// CUDA-core form above spends ~18 instructions per cached element for G = 8 and is bound by them,
+// not by memory.  Here a warp takes 16 slots at a time through mma.sync m16n8k16 (fp32
+// accumulation), the 8 columns being the query heads (zero beyond G), with operands taken
+// straight from 16-byte global loads:
+//   logits  S[16 slots x 8] = K[16 x d] . Q^T: a sum over d does not depend on the order of its
+//           terms, so lane (r, c) = (lane / 4, lane % 4) feeds the elements 32j + 8c .. + 7 of
+//           its rows r and r + 8 (and of query r) as the instruction's k-columns 2c, 2c+1, 2c+8,
+//           2c+9 of chunks 2j and 2j + 1: no shuffle, no shared-memory staging.
+//   output  O^T[d x 8] = V^T[d x 16 slots] . P^T: lane (r, c) loads elements 16r .. 16r + 15
+//           (d = 128) of slots 2c, 2c+1, 2c+8, 2c+9 and interleaves two rows with one byte
+//           permute per register so that a slot pair sits in one register as the instruction
+//           wants; row r / r + 8 of m-tile t is element E*r + t / E*r + E/2 + t (E = d / 8).
+// Probabilities stay fp32 in shared memory for the scores; for the product they are rounded to
+// fp16 (fp16 storage) or split into two bf16 terms hi + lo (bf16 storage, two products), the
+// same precision argument as in the prefill's attention pass.
+template <typename T> struct GroupMma;
+template <> struct GroupMma<__half> {
+    static constexpr int kTerms = 1;
+    __device__ static void mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+    {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    // term 0: the pair rounded to fp16 (there is no second term)
+    __device__ static uint32_t pack(float lo, float hi, int)
+    {
+        const __half2 h = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t *>(&h);
+    }
+};
+template <> struct GroupMma<__nv_bfloat16> {
+    static constexpr int kTerms = 2;
+    __device__ static void mma(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+    {
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+                     "{%0,%1,%2,%3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+    }
+    // term 0: the pair rounded to bf16; term 1: what that rounding left over, again in bf16
+    __device__ static uint32_t pack(float lo, float hi, int term)
+    {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+        if (term == 1) h = __floats2bfloat162_rn(lo - __low2float(h), hi - __high2float(h));
+        return *reinterpret_cast<const uint32_t *>(&h);
+    }
+};
+
+constexpr int kMmaCols = 8;      // query-head columns of the instruction
+
+__host__ __device__ inline size_t group_mma_smem_bytes(int M, int d)
+{
+    // probabilities [wstride][8], partial outputs [warps][8][d], staged scores and positions
+    return ((size_t)(kMmaCols + 2) * group_wstride(M) + (size_t)(kGroupThreads / 32) * kMmaCols * d) * sizeof(float);
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kGroupThreads, 2)
+decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restrict__ q,
+                             const T *__restrict__ k_new, const T *__restrict__ v_new, T *__restrict__ out,
+                             int32_t *__restrict__ evicted)
+{
+    static_assert(sizeof(T) == 2 && (D == 64 || D == 128), "16-bit storage");
+    constexpr int NW = kGroupThreads / 32;
+    constexpr int KL = D / 32;                // 16-byte loads per K row and lane
+    constexpr int E = D / 8;                  // V elements per slot and lane
+    constexpr int VL = E / 8;                 // 16-byte loads per V row and lane
+    constexpr int MT = D / 16;                // m-tiles of the output product
+    using Mma = GroupMma<T>;
+    const int M = c.M;
+    const int wstride = (int)group_wstride(M);
+
+    extern __shared__ __align__(16) float gsm[];
+    float *w = gsm;                                   // [wstride][8] logits, then probabilities
+    float *part = w + (size_t)kMmaCols * wstride;     // [NW][8][D] partial outputs
+    float *s_old = part + (size_t)NW * kMmaCols * D;  // [wstride] the unit's scores before the step
+    int32_t *s_pos = reinterpret_cast<int32_t *>(s_old + wstride);
+    __shared__ float red_m[NW][kMmaCols], red_l[NW][kMmaCols];
+    __shared__ unsigned long long red_key[NW];
+    __shared__ int red_slot[NW];
+    __shared__ int s_target;
+
+    const int u = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int r = lane >> 2, cq = lane & 3;
+    const int cnt = min(c.count[u], M);
+    const int p = c.len[u];
+    T *Ku = reinterpret_cast<T *>(c.K) + (size_t)u * M * D;
+    T *Vu = reinterpret_cast<T *>(c.V) + (size_t)u * M * D;
+    float *Su = c.S + (size_t)u * M;
+    int32_t *posu = c.pos + (size_t)u * M;
+    const T *qu = q + (size_t)u * G * D;              // [G][D]
+    const T *knu = k_new + (size_t)u * D, *vnu = v_new + (size_t)u * D;
+
+    for (int s = tid; s < cnt; s += kGroupThreads) {
+        cp_async4(s_old + s, Su + s);
+        cp_async4(s_pos + s, posu + s);
+    }
+
+    // query r (zero beyond the group), the elements this lane pairs with its K slices
+    uint4 qreg[KL];
+#pragma unroll
+    for (int j = 0; j < KL; ++j) {
+        qreg[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < G) qreg[j] = *reinterpret_cast<const uint4 *>(qu + (size_t)r * D + 32 * j + 8 * cq);
+    }
+
+    const int ntile = (cnt + 1 + 15) >> 4;            // rows 0..cnt-1 cached, row cnt the new token
+    auto row_ptr = [&](int s, const T *base, const T *fresh) { return s < cnt ? base + (size_t)s * D : fresh; };
+
+    // ---- (i) logits ------------------------------------------------------------------------------
+    auto load_k = [&](uint4(&buf)[2][KL], int tile) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int s = tile * 16 + r + 8 * h;
+#pragma unroll
+            for (int j = 0; j < KL; ++j) {
+                buf[h][j] = make_uint4(0u, 0u, 0u, 0u);
+                if (tile < ntile && s <= cnt)
+                    buf[h][j] = *reinterpret_cast<const uint4 *>(row_ptr(s, Ku, knu) + 32 * j + 8 * cq);
+            }
+        }
+    };
+    {
+        uint4 cur[2][KL], nxt[2][KL];
+        load_k(cur, warp);
+        for (int tile = warp; tile < ntile; tile += NW) {
+            load_k(nxt, tile + NW);
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int j = 0; j < KL; ++j) {
+                const uint32_t a_even[4] = {cur[0][j].x, cur[1][j].x, cur[0][j].y, cur[1][j].y};
+                const uint32_t a_odd[4] = {cur[0][j].z, cur[1][j].z, cur[0][j].w, cur[1][j].w};
+                Mma::mma(acc, a_even, qreg[j].x, qreg[j].y);
+                Mma::mma(acc, a_odd, qreg[j].z, qreg[j].w);
+            }
+            // acc: rows r, r + 8 of the tile, query columns 2c and 2c + 1
+            const int s0 = tile * 16 + r;
+            if (s0 <= cnt)
+                *reinterpret_cast<float2 *>(w + (size_t)s0 * kMmaCols + 2 * cq) = make_float2(acc[0] * c.scale, acc[1] * c.scale);
+            if (s0 + 8 <= cnt)
+                *reinterpret_cast<float2 *>(w + (size_t)(s0 + 8) * kMmaCols + 2 * cq) =
+                    make_float2(acc[2] * c.scale, acc[3] * c.scale);
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int j = 0; j < KL; ++j) cur[h][j] = nxt[h][j];
+        }
+    }
+
+    // ---- (iii, loads) the first tile of values is on its way while the softmax runs ---------------
+    auto load_v = [&](uint4(&buf)[4][VL], int tile) {
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int s = tile * 16 + 2 * cq + (x & 1) + 8 * (x >> 1);
+#pragma unroll
+            for (int i = 0; i < VL; ++i) {
+                buf[x][i] = make_uint4(0u, 0u, 0u, 0u);
+                if (tile < ntile && s <= cnt)
+                    buf[x][i] = *reinterpret_cast<const uint4 *>(row_ptr(s, Vu, vnu) + E * r + 8 * i);
+            }
+        }
+    };
+    uint4 vcur[4][VL], vnxt[4][VL];
+    load_v(vcur, warp);
+    __syncthreads();
+
+    // ---- (ii) softmax per query column: thread = (row % 32, column) ------------------------------
+    {
+        const int g = tid & 7;
+        const int nrow = cnt + 1;
+        float m = -INFINITY;
+        if (g < G)
+            for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) m = fmaxf(m, w[s * kMmaCols + g]);
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
+        if (lane < 8) red_m[warp][lane] = m;
+        __syncthreads();
+        m = red_m[0][g];
+#pragma unroll
+        for (int x = 1; x < NW; ++x) m = fmaxf(m, red_m[x][g]);
+        float l = 0.f;
+        if (g < G)
+            for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) {
+                const float e = expf(w[s * kMmaCols + g] - m);
+                w[s * kMmaCols + g] = e;
+                l += e;
+            }
+        l += __shfl_xor_sync(0xffffffffu, l, 8);
+        l += __shfl_xor_sync(0xffffffffu, l, 16);
+        if (lane < 8) red_l[warp][lane] = l;
+        __syncthreads();
+        l = red_l[0][g];
+#pragma unroll
+        for (int x = 1; x < NW; ++x) l += red_l[x][g];                  // fixed order
+        const float inv = 1.f / l;
+        for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8)
+            w[s * kMmaCols + g] = g < G ? w[s * kMmaCols + g] * inv : 0.f;   // probabilities; unused columns 0
+    }
+    __syncthreads();
+
+    // ---- (iii) out^T[d x 8] = sum over slots V^T . P^T ----------------------------------------------
+    float oacc[MT][4];
+#pragma unroll
+    for (int t = 0; t < MT; ++t)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) oacc[t][e] = 0.f;
+    for (int tile = warp; tile < ntile; tile += NW) {
+        load_v(vnxt, tile + NW);
+        // P^T fragment: slots 2c, 2c+1 (b0) and 2c+8, 2c+9 (b1) of the tile, query r
+        float pf[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const int s = tile * 16 + 2 * cq + (x & 1) + 8 * (x >> 1);
+            pf[x] = s <= cnt ? w[(size_t)s * kMmaCols + r] : 0.f;
+        }
+#pragma unroll
+        for (int term = 0; term < Mma::kTerms; ++term) {
+            const uint32_t b0 = Mma::pack(pf[0], pf[1], term), b1 = Mma::pack(pf[2], pf[3], term);
+#pragma unroll
+            for (int t = 0; t < MT; ++t) {
+                // element E*r + t (rows r) and E*r + E/2 + t (rows r + 8) of the four slots
+                const uint32_t *v0 = reinterpret_cast<const uint32_t *>(vcur[0]);
+                const uint32_t *v1 = reinterpret_cast<const uint32_t *>(vcur[1]);
+                const uint32_t *v2 = reinterpret_cast<const uint32_t *>(vcur[2]);
+                const uint32_t *v3 = reinterpret_cast<const uint32_t *>(vcur[3]);
+                const int lo = t >> 1, hi = (E / 2 + t) >> 1;
+                const uint32_t sel = (t & 1) ? 0x7632u : 0x5410u;
+                const uint32_t a[4] = {__byte_perm(v0[lo], v1[lo], sel), __byte_perm(v0[hi], v1[hi], sel),
+                                       __byte_perm(v2[lo], v3[lo], sel), __byte_perm(v2[hi], v3[hi], sel)};
+                Mma::mma(oacc[t], a, b0, b1);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int i = 0; i < VL; ++i) vcur[x][i] = vnxt[x][i];
+    }
+    // oacc[t]: (element E*r + t, queries 2c, 2c+1), (element E*r + E/2 + t, queries 2c, 2c+1)
+#pragma unroll
+    for (int t = 0; t < MT; ++t) {
+        float *pw = part + (size_t)warp * kMmaCols * D;
+        pw[(2 * cq) * D + E * r + t] = oacc[t][0];
+        pw[(2 * cq + 1) * D + E * r + t] = oacc[t][1];
+        pw[(2 * cq) * D + E * r + E / 2 + t] = oacc[t][2];
+        pw[(2 * cq + 1) * D + E * r + E / 2 + t] = oacc[t][3];
+    }
+    cp_async_wait_all();                       // this thread's staged scores and positions
+    __syncthreads();
+    for (int x = tid; x < G * D; x += kGroupThreads) {
+        float o = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < NW; ++wv) o += part[(size_t)wv * kMmaCols * D + x];
+        out[(size_t)u * G * D + x] = Elem<T>::from_float(o);
+    }
+
+    // ---- (iv) S <- alpha*S + sum_g a_g ; candidates for eviction ---------------------------------
+    const bool full = cnt >= M;
+    const int newest_evictable = p - c.R;
+    unsigned long long best = ~0ull;
+    int best_slot = -1;
+    for (int s = tid; s < cnt; s += kGroupThreads) {
+        float gain = 0.f;
+        for (int g = 0; g < G; ++g) gain += w[(size_t)s * kMmaCols + g];
+        const float sn = fmaf(alpha, s_old[s], gain);
+        Su[s] = sn;
+        const int ps = s_pos[s];
+        if (full && ps <= newest_evictable) {
+            const unsigned long long key = ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
+            if (key < best) { best = key; best_slot = s; }
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int os = __shfl_xor_sync(0xffffffffu, best_slot, o);
+        if (ob < best) { best = ob; best_slot = os; }
+    }
+    if (lane == 0) { red_key[warp] = best; red_slot[warp] = best_slot; }
+    __syncthreads();
+
+    // ---- (v) eviction and in-place insert, (vi) length ------------------------------------------
+    float s_new = 0.f;
+    for (int g = 0; g < G; ++g) s_new += w[(size_t)cnt * kMmaCols + g];
+    if (tid == 0) {
+        int target = full ? -2 : cnt;
+        if (full) {
+            unsigned long long gb = red_key[0];
+            int gs = red_slot[0];
+            for (int x = 1; x < NW; ++x)
+                if (red_key[x] < gb) { gb = red_key[x]; gs = red_slot[x]; }
+            const unsigned long long self_key = ((unsigned long long)__float_as_uint(s_new) << 32) | (unsigned)p;
+            if (gs >= 0 && (c.R > 0 || gb < self_key)) target = gs;
+        }
+        s_target = target;
+    }
+    __syncthreads();
+    const int target = s_target;
+    if (target >= 0) {
+        constexpr int LPR = D / 8;
+        if (tid < LPR)
+            *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * 8) =
+                *reinterpret_cast<const uint4 *>(knu + tid * 8);
+        else if (tid < 2 * LPR)
+            *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * 8) =
+                *reinterpret_cast<const uint4 *>(vnu + (tid - LPR) * 8);
+    }
+    if (tid == 0) {
+        if (target >= 0) {
+            Su[target] = s_new;
+            posu[target] = p;
+        }
+        if (!full) c.count[u] = cnt + 1;
+        c.len[u] = p + 1;
+        evicted[u] = full ? target : -1;
+    }
+}
+
+template <typename T, int D>
+cudaError_t launch_group_mma(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
+                             const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
+{
+    const size_t smem = group_mma_smem_bytes(c.M, D);
+    auto kern = decode_step_group_mma_kernel<T, D>;
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    kern<<<c.U, kGroupThreads, smem, s>>>(c, G, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
+                                           static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
+    count_launch();
+    return cudaGetLastError();
+}
+
 template <typename T, int D, int GMAX>
 cudaError_t launch_group_n(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
                            const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
@@ -336,6 +673,11 @@ template <typename T, int D>
 cudaError_t launch_group(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
                          const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
+    // 16-bit storage takes the tensor-core form whenever its shared memory fits
+    if constexpr (sizeof(T) == 2) {
+        if (group_mma_smem_bytes(c.M, D) <= 220 * 1024)
+            return launch_group_mma<T, D>(c, G, alpha, q, k_new, v_new, out, evicted, s);
+    }
     if (G <= 2) return launch_group_n<T, D, 2>(c, G, alpha, q, k_new, v_new, out, evicted, s);
     if (G <= 4) return launch_group_n<T, D, 4>(c, G, alpha, q, k_new, v_new, out, evicted, s);
     return launch_group_n<T, D, 8>(c, G, alpha, q, k_new, v_new, out, evicted, s);
