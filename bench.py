@@ -373,9 +373,72 @@ def run_ours(args):
             decode_layer_rotation(a2sf, dev, name, layers, args.rotation_steps, args.rotation_reps)
             for name, layers in (("llama2_7b", 32), ("opt_6p7b", 32), ("long_context", 32),
                                  ("llama2_13b", 1))]          # the headline workload, graph-replayed
+    if rank == 0 and world == 1 and not args.no_grouped:
+        # grouped query heads (not part of the headline): the same policy on 8 K/V heads per row
+        result["decode_grouped"] = [decode_grouped(a2sf, dev, G, 8, args.rotation_steps, args.rotation_reps)
+                                    for G in (4, 8)]
     if rank == 0:
         print(json.dumps(result))
     a2dist.finalize()
+
+
+def decode_grouped(a2sf, dev, G, layers, steps, reps):
+    """Grouped-query decode step (G query heads per K/V head, one pruned cache per K/V head) on the
+    headline workload's policy with 8 K/V heads per batch row: 256 units x 512 slots, 69 MB per
+    launch.  Timed like `decode_layer_rotation`: one layer (fits in L2) and `layers` caches stepped
+    round-robin (larger than L2), `steps` x layers launches replayed from a CUDA graph."""
+    w = wl.WORKLOADS["llama2_13b"].scaled(H=8, n=1024)
+    wq = w.scaled(H=w.H * G)
+    q = wl.make_prompt(wq, dev)[0]
+    _, k, v = wl.make_prompt(w, dev)
+    dq = wl.make_decode(wq, dev, t_range=(0, steps))[0]
+    _, dk, dv = wl.make_decode(w, dev, t_range=(0, steps))
+    p = a2sf.make_params(w.B, w.H, w.d, w.torch_dtype, w.budget, w.recent, w.alpha)
+    _, S, kept, _ = a2sf.a2sf_prefill_group(p, G, q, k, v)
+    del q
+    # K and V once per unit, whatever the group size; the G query and output rows on top
+    bytes_per_launch = w.units * (w.decode_bytes_per_unit_step() + (G - 1) * 2 * w.d * 2)
+    res = {"workload": f"B{w.B} Hkv{w.H} group{G} d{w.d} alpha{w.alpha} budget{w.budget} recent{w.recent} bf16",
+           "bytes_per_launch": bytes_per_launch, "steps_per_replay": steps, "repetitions": reps}
+    for L in sorted({1, layers}):
+        caches = [a2sf.Cache(p, dev) for _ in range(L)]
+        o = torch.empty((L, w.B, w.H * G, w.d), dtype=w.torch_dtype, device=dev)
+        e = torch.empty((L, w.B, w.H), dtype=torch.int32, device=dev)
+
+        def restore():
+            for c in caches:
+                c.a2sf_cache_load(k, v, S, kept)
+
+        def run():
+            for t in range(steps):
+                for l, c in enumerate(caches):
+                    c.a2sf_decode_step_group(G, w.alpha, dq[t], dk[t], dv[t], o[l], e[l])
+
+        restore(); run()                        # kernel attributes are set outside the capture
+        torch.cuda.synchronize()
+        restore()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            run()
+        times = []
+        for _ in range(reps):
+            restore()
+            ev = cuda_events(2)
+            ev[0].record(); g.replay(); ev[1].record()
+            torch.cuda.synchronize()
+            times.append(ev[0].elapsed_time(ev[1]) * 1e3 / (steps * L))      # us per launch
+        assert a2sf.a2sf_last_device_status() == a2sf.A2SF_OK
+        med, best = statistics.median(times), min(times)
+        res["layers_%d" % L] = {
+            "working_set_mb": L * bytes_per_launch / 1e6,
+            "l2": "larger_than_l2" if L * bytes_per_launch > 126e6 else "l2_resident",
+            "us_per_launch_median": med, "us_per_launch_min": best,
+            "gbps_median": bytes_per_launch / med / 1e3, "gbps_max": bytes_per_launch / best / 1e3}
+        del g
+        for c in caches:
+            c.close()
+    return res
 
 
 def decode_layer_rotation(a2sf, dev, name, layers, steps, reps):
@@ -556,6 +619,7 @@ def main():
                     help="skip the separate timing of the row-by-row streamed prompt")
     ap.add_argument("--no-rotation", action="store_true",
                     help="skip the layer-rotation decode timing of the L2-resident workloads")
+    ap.add_argument("--no-grouped", action="store_true", help="skip the grouped-query decode timing")
     ap.add_argument("--rotation-steps", type=int, default=16, help="decode steps per graph replay")
     ap.add_argument("--rotation-reps", type=int, default=10)
     args = ap.parse_args()

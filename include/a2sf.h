@@ -274,8 +274,9 @@ int a2sf_decode_multi(a2sf_cache *cache, float alpha, int32_t steps,
  * (a2sf_cache_load).  q, out DEVICE [B][H*group][d] contiguous; k_new, v_new DEVICE [B][H][d];
  * evicted_slot [B][H].  Each query head attends over the cached tokens and the new one; the
  * cached scores become alpha * S + sum_g a_g, the new token's score sum_g a_g,self; eviction as
- * in a2sf_decode_step.  A2SF_ERR_UNSUPPORTED when group > A2SF_MAX_GROUP or group * budget is
- * too large for one CTA's shared memory (about 50,000 slots x heads).
+ * in a2sf_decode_step.  A2SF_ERR_UNSUPPORTED when group > A2SF_MAX_GROUP or (group + 2) * budget
+ * is too large for one CTA's shared memory (about 47,000 for d = 128, group = 8).  For 16-bit
+ * storage the products of the group run on the tensor cores (fp32 accumulation).
  * ------------------------------------------------------------------------- */
 #define A2SF_MAX_GROUP 8
 size_t a2sf_prefill_group_workspace_bytes(const a2sf_params *p, int32_t group, int32_t n);

@@ -414,11 +414,17 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     ("opt_6p7b", dict(B=2, H=1, n=300, budget=64, recent=0, steps=40, alpha=0.7), 8),   # fp16, all selective
     ("tiny_fp32", dict(H=3, n=150, steps=24), 2),                                  # fp32 d = 64, CUDA cores
     ("llama2_7b", dict(H=2, n=40, budget=64, recent=32, steps=40), 3),             # appends, then evicts
-    # 64 units and more take the persistent streaming kernel with G queries per unit
+    # many units at once: every SM holds one or two of the one-CTA-per-unit kernels
     ("llama2_7b", dict(B=8, H=8, n=160, budget=96, recent=48, steps=24), 4),
     ("opt_6p7b", dict(B=9, H=8, n=140, budget=70, recent=0, steps=16), 8),
     ("tiny_fp32", dict(B=16, H=5, n=100, budget=40, recent=20, steps=12), 2),
     ("llama2_13b", dict(B=4, H=16, n=130, budget=300, recent=100, steps=12, d=64), 5),   # appends only, d = 64
+    # 16-bit storage runs the group's products on the tensor cores, fp32 storage on CUDA cores
+    # (instantiated for group bounds 2, 4 and 8): a ragged last tile of slots, d = 64, a group of one
+    ("opt_6p7b", dict(B=1, H=3, n=200, budget=77, recent=30, steps=30, d=64), 6),
+    ("llama2_7b", dict(B=1, H=2, n=300, budget=130, recent=65, steps=30), 1),
+    ("tiny_fp32", dict(H=2, n=150, steps=24), 4),
+    ("tiny_fp32", dict(B=2, H=2, n=90, budget=40, recent=0, steps=20), 7),
 ])
 def test_grouped_query_heads_against_the_oracle(name, kw, G):
     import oracle
