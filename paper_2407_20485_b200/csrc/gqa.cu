@@ -491,8 +491,10 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
         const int g = tid & 7;
         const int nrow = cnt + 1;
         float m = -INFINITY;
-        if (g < G)
+        if (g < G) {
+#pragma unroll 4
             for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) m = fmaxf(m, w[s * kMmaCols + g]);
+        }
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
         m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
         if (lane < 8) red_m[warp][lane] = m;
@@ -502,6 +504,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
         for (int x = 1; x < NW; ++x) m = fmaxf(m, red_m[x][g]);
         float l = 0.f;
         if (g < G)
+#pragma unroll 4
             for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) {
                 const float e = expf(w[s * kMmaCols + g] - m);
                 w[s * kMmaCols + g] = e;
@@ -515,6 +518,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
 #pragma unroll
         for (int x = 1; x < NW; ++x) l += red_l[x][g];                  // fixed order
         const float inv = 1.f / l;
+#pragma unroll 4
         for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8)
             w[s * kMmaCols + g] = g < G ? w[s * kMmaCols + g] * inv : 0.f;   // probabilities; unused columns 0
     }
