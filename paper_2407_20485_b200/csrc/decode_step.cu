@@ -78,7 +78,7 @@ struct SplitExchange {
 };
 
 template <typename T, int D, int NT>
-__global__ void __launch_bounds__(NT)
+__global__ void __launch_bounds__(NT, 2)
 decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__ alpha_vec,
                          const T *__restrict__ q, const T *__restrict__ k_new,
                          const T *__restrict__ v_new, T *__restrict__ out, int32_t *__restrict__ evicted)
@@ -125,19 +125,49 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     float qf[VEC];
     Elem<T>::unpack(*reinterpret_cast<const uint4 *>(q + uo + sub * VEC), qf);
 
-    // ---- (i) logits of the slice, and (rank 0) of the new key ---------------------------------
-    const int ngroups = (nloc + RPW - 1) / RPW;
-    for (int g = warp; g < ngroups; g += NW * kUnroll) {
-        uint4 r[kUnroll];
+    // The step is a chain of dependent phases around little data per CTA, so every global word is
+    // requested as early as it can be.  Rows move in batches of kBatchRows per CTA through two
+    // register buffers: two batches are in flight at any time, the first two batches of V are
+    // requested as soon as the last K batches have been consumed (they travel while the CTA sits
+    // in the softmax reductions), and this thread's scores and positions are requested here.
+    constexpr int kU = 8;                         // 16-byte loads per lane and batch
+    constexpr int kBatchRows = NW * RPW * kU;
+    constexpr int kPre = 2;                       // score/position words preloaded per thread
+    float s_pre[kPre];
+    int p_pre[kPre];
 #pragma unroll
-        for (int x = 0; x < kUnroll; ++x) {
-            const int row = (g + x * NW) * RPW + rsel;
-            r[x] = make_uint4(0, 0, 0, 0);
-            if (row < nloc) r[x] = ld_stream16(Ku + (size_t)(s0 + row) * D + sub * VEC);
+    for (int i = 0; i < kPre; ++i) {
+        const int s = tid + i * NT;
+        s_pre[i] = 0.f;
+        p_pre[i] = 0;
+        if (s < nloc) {
+            s_pre[i] = Su[s0 + s];
+            p_pre[i] = posu[s0 + s];
         }
+    }
+    const int nb = ((nloc + kBatchRows - 1) / kBatchRows + 1) & ~1;     // batches, padded to even
+    auto load_batch = [&](uint4(&r)[kU], const T *base, int bidx) {
 #pragma unroll
-        for (int x = 0; x < kUnroll; ++x) {
-            const int row = (g + x * NW) * RPW + rsel;
+        for (int x = 0; x < kU; ++x) {
+            const int row = ((bidx * kU + x) * NW + warp) * RPW + rsel;
+            r[x] = make_uint4(0, 0, 0, 0);
+            if (bidx < nb && row < nloc) r[x] = ld_stream16(base + (size_t)(s0 + row) * D + sub * VEC);
+        }
+    };
+    // batch index b: K batch b for b < nb, V batch b - nb after that
+    auto load_next = [&](uint4(&r)[kU], int b) {
+        if (b < nb) load_batch(r, Ku, b);
+        else load_batch(r, Vu, b - nb);
+    };
+    uint4 ra[kU], rb[kU];
+    load_batch(ra, Ku, 0);
+    load_batch(rb, Ku, 1);
+
+    // ---- (i) logits of the slice, and (rank 0) of the new key ---------------------------------
+    auto logits_of = [&](const uint4(&r)[kU], int bidx) {
+#pragma unroll
+        for (int x = 0; x < kU; ++x) {
+            const int row = ((bidx * kU + x) * NW + warp) * RPW + rsel;
             float kf[VEC];
             Elem<T>::unpack(r[x], kf);
             float dot = 0.f;
@@ -147,6 +177,12 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
             for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
             if (sub == 0 && row < nloc) w[row] = dot * c.scale;
         }
+    };
+    for (int b = 0; b < nb; b += 2) {
+        logits_of(ra, b);
+        load_next(ra, b + 2);
+        logits_of(rb, b + 1);
+        load_next(rb, b + 3);
     }
     if (warp == 0 && rank == 0) {
         float kf[VEC];
@@ -176,23 +212,23 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-    for (int g = warp; g < ngroups; g += NW * kUnroll) {
-        uint4 r[kUnroll];
+    auto accumulate = [&](const uint4(&r)[kU], int bidx) {
 #pragma unroll
-        for (int x = 0; x < kUnroll; ++x) {
-            const int row = (g + x * NW) * RPW + rsel;
-            r[x] = make_uint4(0, 0, 0, 0);
-            if (row < nloc) r[x] = ld_stream16(Vu + (size_t)(s0 + row) * D + sub * VEC);
-        }
-#pragma unroll
-        for (int x = 0; x < kUnroll; ++x) {
-            const int row = (g + x * NW) * RPW + rsel;
+        for (int x = 0; x < kU; ++x) {
+            const int row = ((bidx * kU + x) * NW + warp) * RPW + rsel;
             const float ws = row < nloc ? w[row] : 0.f;
             float vf[VEC];
             Elem<T>::unpack(r[x], vf);
 #pragma unroll
             for (int e = 0; e < VEC; ++e) acc[e] = fmaf(ws, vf[e], acc[e]);
         }
+    };
+    // V batches 0 and 1 are already in ra and rb (nb is even)
+    for (int b = 0; b < nb; b += 2) {
+        accumulate(ra, b);
+        load_batch(ra, Vu, b + 2);
+        accumulate(rb, b + 1);
+        load_batch(rb, Vu, b + 3);
     }
 #pragma unroll
     for (int o = LPR; o < 32; o <<= 1)
@@ -235,18 +271,21 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     const float rescale = expf(m_loc - m);
     unsigned long long best = ~0ull;
     int best_slot = -1;
-    for (int s = tid; s < nloc; s += NT) {
+    auto update = [&](int s, float s_before, int ps) {
         const float a = w[s] * rescale / l;
-        const float sn = fmaf(alpha, Su[s0 + s], a);
+        const float sn = fmaf(alpha, s_before, a);
         Su[s0 + s] = sn;
-        const int ps = posu[s0 + s];
         if (full && ps <= newest_evictable) {
             // scores are >= 0, so their bit patterns order like the values
             const unsigned long long key =
                 ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
             if (key < best) { best = key; best_slot = s0 + s; }
         }
-    }
+    };
+#pragma unroll
+    for (int i = 0; i < kPre; ++i)
+        if (tid + i * NT < nloc) update(tid + i * NT, s_pre[i], p_pre[i]);
+    for (int s = tid + kPre * NT; s < nloc; s += NT) update(s, Su[s0 + s], posu[s0 + s]);
     // positions are distinct, so the minimum key identifies its slot
     for (int o = 16; o > 0; o >>= 1) {
         const unsigned long long ob = __shfl_xor_sync(0xffffffffu, best, o);
