@@ -32,7 +32,6 @@ int *decode_status_word()
 
 constexpr int kDecodeThreads = 256;
 constexpr int kSplitMinBudget = 512;         // split-K only pays for long caches
-constexpr int kUnroll = 4;
 
 template <int NT>
 __device__ __forceinline__ float block_max(float v, float *red)
@@ -64,18 +63,35 @@ __device__ __forceinline__ float block_sum(float v, float *red)
 // Split-K variant for few units with large budgets (flash-decoding): a thread-block cluster of
 // C CTAs shares one unit, each CTA owning a contiguous slice of its slots.  Every CTA computes
 // the logits, the local maximum, the local exponential sum and the unnormalised partial output
-// of its slice; the partials meet in distributed shared memory: all CTAs read every (max, sum)
-// pair to form the global softmax constants, rank 0 combines the partial outputs, every CTA
-// then updates the scores of its own slots and publishes its local eviction candidate, and
-// rank 0 picks the global (score, position) minimum and writes the new token in place.
+// of its slice; the partials meet in distributed shared memory: every CTA stores its (max, sum)
+// pair into all CTAs' inboxes and its partial output into rank 0's, one cluster barrier later
+// each CTA forms the global softmax constants from its own inbox and rank 0 combines the
+// outputs; every CTA then updates the scores of its own slots, stores its local eviction
+// candidate into rank 0's inbox, arrives at the second barrier and is done; rank 0 alone waits
+// there, picks the global (score, position) minimum and writes the new token in place.
+// A peer's shared memory may be written only once that CTA runs: every thread arrives at a
+// first barrier when the kernel starts and waits for it just before its first remote store,
+// by which time it has long completed.
 // With C = 1 this is the plain one-CTA-per-unit kernel.
 // ============================================================================================
-struct SplitExchange {
-    float m, l;                    // local maximum and sum of exp(logit - m)
-    unsigned long long best;       // local (bits(S) << 32 | position) minimum over evictable slots
-    int best_slot;
-    float out[128];                // unnormalised partial output (relative to m)
+constexpr int kMaxSplit = 8;       // CTAs per unit at most
+// What the CTAs of a cluster hand to each other, indexed by the sender's rank.  Every CTA
+// receives all (max, sum) pairs; only rank 0's copy of the rest is ever written.
+struct SplitInbox {
+    float m[kMaxSplit], l[kMaxSplit];          // local maximum and sum of exp(logit - m)
+    unsigned long long best[kMaxSplit];        // local (bits(S) << 32 | position) minimum over evictable slots
+    int best_slot[kMaxSplit];
+    float out[kMaxSplit][128];                 // unnormalised partial outputs (relative to m)
 };
+
+__device__ __forceinline__ void cluster_arrive()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait()
+{
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 template <typename T, int D, int NT>
 __global__ void __launch_bounds__(NT, 2)
@@ -92,6 +108,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     cg::cluster_group cluster = cg::this_cluster();
     const int C = (int)cluster.num_blocks();
     const int rank = (int)cluster.block_rank();
+    cluster_arrive();                            // "this CTA runs": waited for before the first remote store
 
     extern __shared__ float smem[];
     const int M = c.M;
@@ -99,7 +116,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     float *w = smem;                             // [per_max+1] logits, then exp(logit - max)
     float *part = w + ((per_max + 1 + 3) & ~3);  // [NW][D] partial outputs
     float *red = part + NW * D;                  // [NW] reduction scratch
-    __shared__ SplitExchange xch;
+    __shared__ SplitInbox inbox;
     __shared__ unsigned long long red_key[NW];
     __shared__ int red_slot[NW];
     __shared__ int s_target;
@@ -238,30 +255,30 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
 #pragma unroll
         for (int e = 0; e < VEC; ++e) part[warp * D + sub * VEC + e] = acc[e];
     __syncthreads();
+    cluster_wait();                              // every CTA of the cluster runs
     if (tid < D) {
         float o = 0.f;
 #pragma unroll
         for (int x = 0; x < NW; ++x) o += part[x * D + tid];
         if (rank == 0) o = fmaf(w[nloc], Elem<T>::to_float(v_new[uo + tid]), o);
-        xch.out[tid] = o;
+        cluster.map_shared_rank(&inbox, 0)->out[rank][tid] = o;
     }
-    if (tid == 0) { xch.m = m_loc; xch.l = l_loc; }
-    cluster.sync();
+    if (tid < C) {
+        SplitInbox *peer = cluster.map_shared_rank(&inbox, tid);
+        peer->m[rank] = m_loc;
+        peer->l[rank] = l_loc;
+    }
+    cluster_arrive();
+    cluster_wait();
 
-    // ---- global softmax constants: every CTA reads every (max, sum) pair, in rank order ----------
+    // ---- global softmax constants from the (max, sum) pairs, in rank order ------------------------
     float m = -INFINITY;
-    for (int r2 = 0; r2 < C; ++r2) m = fmaxf(m, cluster.map_shared_rank(&xch, r2)->m);
+    for (int r2 = 0; r2 < C; ++r2) m = fmaxf(m, inbox.m[r2]);
     float l = 0.f;
-    for (int r2 = 0; r2 < C; ++r2) {
-        const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
-        l += x->l * expf(x->m - m);          // an empty slice has m = -inf, l = 0
-    }
+    for (int r2 = 0; r2 < C; ++r2) l += inbox.l[r2] * expf(inbox.m[r2] - m);   // an empty slice has m = -inf, l = 0
     if (rank == 0 && tid < D) {
         float o = 0.f;
-        for (int r2 = 0; r2 < C; ++r2) {
-            const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
-            o = fmaf(x->out[tid], expf(x->m - m), o);
-        }
+        for (int r2 = 0; r2 < C; ++r2) o = fmaf(inbox.out[r2][tid], expf(inbox.m[r2] - m), o);
         out[uo + tid] = Elem<T>::from_float(o / l);
     }
 
@@ -299,51 +316,48 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         int gs = red_slot[0];
         for (int x = 1; x < NW; ++x)
             if (red_key[x] < gb) { gb = red_key[x]; gs = red_slot[x]; }
-        xch.best = gb;
-        xch.best_slot = gs;
+        SplitInbox *root = cluster.map_shared_rank(&inbox, 0);
+        root->best[rank] = gb;
+        root->best_slot[rank] = gs;
     }
-    cluster.sync();
+    cluster_arrive();
+    if (rank != 0) return;                       // nobody reads this CTA's shared memory
+    cluster_wait();
 
     // ---- (v) rank 0 picks the global minimum and inserts the new token in place -------------------
-    if (rank == 0) {
-        const float a_self = w[nloc] * rescale / l;
-        if (tid == 0) {
-            int target = full ? -2 : cnt;
-            if (full) {
-                unsigned long long gb = ~0ull;
-                int gs = -1;
-                for (int r2 = 0; r2 < C; ++r2) {
-                    const SplitExchange *x = cluster.map_shared_rank(&xch, r2);
-                    if (x->best < gb) { gb = x->best; gs = x->best_slot; }
-                }
-                const unsigned long long self_key =
-                    ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
-                if (gs >= 0 && (c.R > 0 || gb < self_key)) target = gs;
-            }
-            s_target = target;
+    const float a_self = w[nloc] * rescale / l;
+    if (tid == 0) {
+        int target = full ? -2 : cnt;
+        if (full) {
+            unsigned long long gb = ~0ull;
+            int gs = -1;
+            for (int r2 = 0; r2 < C; ++r2)
+                if (inbox.best[r2] < gb) { gb = inbox.best[r2]; gs = inbox.best_slot[r2]; }
+            const unsigned long long self_key =
+                ((unsigned long long)__float_as_uint(a_self) << 32) | (unsigned)p;
+            if (gs >= 0 && (c.R > 0 || gb < self_key)) target = gs;
         }
-        __syncthreads();
-        const int target = s_target;
-        if (target >= 0) {
-            if (tid < LPR)
-                *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
-                    *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
-            else if (tid < 2 * LPR)
-                *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
-                    *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
-        }
-        if (tid == 0) {
-            if (target >= 0) {
-                Su[target] = a_self;
-                posu[target] = p;
-            }
-            if (!full) c.count[u] = cnt + 1;
-            c.len[u] = p + 1;
-            evicted[u] = full ? target : -1;
-        }
+        s_target = target;
     }
-    // peers must stay resident until rank 0 has read their shared memory
-    cluster.sync();
+    __syncthreads();
+    const int target = s_target;
+    if (target >= 0) {
+        if (tid < LPR)
+            *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
+                *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
+        else if (tid < 2 * LPR)
+            *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
+                *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
+    }
+    if (tid == 0) {
+        if (target >= 0) {
+            Su[target] = a_self;
+            posu[target] = p;
+        }
+        if (!full) c.count[u] = cnt + 1;
+        c.len[u] = p + 1;
+        evicted[u] = full ? target : -1;
+    }
 }
 
 
