@@ -425,6 +425,9 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     ("llama2_7b", dict(B=1, H=2, n=300, budget=130, recent=65, steps=30), 1),
     ("tiny_fp32", dict(H=2, n=150, steps=24), 4),
     ("tiny_fp32", dict(B=2, H=2, n=90, budget=40, recent=0, steps=20), 7),
+    # a budget whose eight probability columns no longer fit in shared memory: 16-bit storage
+    # falls back to the CUDA-core form
+    ("llama2_7b", dict(B=1, H=1, n=6100, budget=6000, recent=3000, steps=6), 2),
 ])
 def test_grouped_query_heads_against_the_oracle(name, kw, G):
     import oracle
