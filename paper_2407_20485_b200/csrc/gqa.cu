@@ -396,7 +396,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     float *part = w + (size_t)kMmaCols * wstride;     // [NW][8][D] partial outputs
     float *s_old = part + (size_t)NW * kMmaCols * D;  // [wstride] the unit's scores before the step
     int32_t *s_pos = reinterpret_cast<int32_t *>(s_old + wstride);
-    __shared__ float red_m[NW][kMmaCols], red_l[NW][kMmaCols];
+    __shared__ float red_m[NW][kMmaCols], red_l[NW][kMmaCols], s_inv[kMmaCols];
     __shared__ unsigned long long red_key[NW];
     __shared__ int red_slot[NW];
     __shared__ int s_target;
@@ -445,6 +445,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     {
         uint4 cur[2][KL], nxt[2][KL];
         load_k(cur, warp);
+        float mx0 = -INFINITY, mx1 = -INFINITY;      // running maxima of query columns 2c, 2c + 1
         for (int tile = warp; tile < ntile; tile += NW) {
             load_k(nxt, tile + NW);
             float acc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -457,15 +458,32 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
             }
             // acc: rows r, r + 8 of the tile, query columns 2c and 2c + 1
             const int s0 = tile * 16 + r;
-            if (s0 <= cnt)
-                *reinterpret_cast<float2 *>(w + (size_t)s0 * kMmaCols + 2 * cq) = make_float2(acc[0] * c.scale, acc[1] * c.scale);
-            if (s0 + 8 <= cnt)
-                *reinterpret_cast<float2 *>(w + (size_t)(s0 + 8) * kMmaCols + 2 * cq) =
-                    make_float2(acc[2] * c.scale, acc[3] * c.scale);
+            if (s0 <= cnt) {
+                const float2 lg = make_float2(acc[0] * c.scale, acc[1] * c.scale);
+                *reinterpret_cast<float2 *>(w + (size_t)s0 * kMmaCols + 2 * cq) = lg;
+                mx0 = fmaxf(mx0, lg.x);
+                mx1 = fmaxf(mx1, lg.y);
+            }
+            if (s0 + 8 <= cnt) {
+                const float2 lg = make_float2(acc[2] * c.scale, acc[3] * c.scale);
+                *reinterpret_cast<float2 *>(w + (size_t)(s0 + 8) * kMmaCols + 2 * cq) = lg;
+                mx0 = fmaxf(mx0, lg.x);
+                mx1 = fmaxf(mx1, lg.y);
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h)
 #pragma unroll
                 for (int j = 0; j < KL; ++j) cur[h][j] = nxt[h][j];
+        }
+        // the warp's column maxima (over the lanes' rows r): no separate pass over the logits
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+        }
+        if (lane < 4) {
+            red_m[warp][2 * lane] = mx0;
+            red_m[warp][2 * lane + 1] = mx1;
         }
     }
 
@@ -487,42 +505,32 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     __syncthreads();
 
     // ---- (ii) softmax per query column: thread = (row % 32, column) ------------------------------
+    // The exponentials stay unnormalised: the output rows and the scores take the factor 1 / sum
+    // at the end, so the logits are passed over once, between two barriers.
     {
         const int g = tid & 7;
         const int nrow = cnt + 1;
-        float m = -INFINITY;
-        if (g < G) {
-#pragma unroll 4
-            for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) m = fmaxf(m, w[s * kMmaCols + g]);
-        }
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 8));
-        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 16));
-        if (lane < 8) red_m[warp][lane] = m;
-        __syncthreads();
-        m = red_m[0][g];
+        float m = red_m[0][g];
 #pragma unroll
         for (int x = 1; x < NW; ++x) m = fmaxf(m, red_m[x][g]);
         float l = 0.f;
-        if (g < G)
 #pragma unroll 4
-            for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) {
-                const float e = expf(w[s * kMmaCols + g] - m);
-                w[s * kMmaCols + g] = e;
-                l += e;
-            }
+        for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) {
+            const float e = g < G ? expf(w[s * kMmaCols + g] - m) : 0.f;   // unused columns 0
+            w[s * kMmaCols + g] = e;
+            l += e;
+        }
         l += __shfl_xor_sync(0xffffffffu, l, 8);
         l += __shfl_xor_sync(0xffffffffu, l, 16);
         if (lane < 8) red_l[warp][lane] = l;
-        __syncthreads();
-        l = red_l[0][g];
-#pragma unroll
-        for (int x = 1; x < NW; ++x) l += red_l[x][g];                  // fixed order
-        const float inv = 1.f / l;
-#pragma unroll 4
-        for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8)
-            w[s * kMmaCols + g] = g < G ? w[s * kMmaCols + g] * inv : 0.f;   // probabilities; unused columns 0
     }
     __syncthreads();
+    if (tid < kMmaCols) {
+        float l = red_l[0][tid];
+#pragma unroll
+        for (int x = 1; x < NW; ++x) l += red_l[x][tid];                // fixed order
+        s_inv[tid] = tid < G ? 1.f / l : 0.f;     // read after the barrier that follows the products
+    }
 
     // ---- (iii) out^T[d x 8] = sum over slots V^T . P^T ----------------------------------------------
     float oacc[MT][4];
@@ -576,7 +584,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
         float o = 0.f;
 #pragma unroll
         for (int wv = 0; wv < NW; ++wv) o += part[(size_t)wv * kMmaCols * D + x];
-        out[(size_t)u * G * D + x] = Elem<T>::from_float(o);
+        out[(size_t)u * G * D + x] = Elem<T>::from_float(o * s_inv[x / D]);
     }
 
     // ---- (iv) S <- alpha*S + sum_g a_g ; candidates for eviction ---------------------------------
@@ -586,7 +594,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     int best_slot = -1;
     for (int s = tid; s < cnt; s += kGroupThreads) {
         float gain = 0.f;
-        for (int g = 0; g < G; ++g) gain += w[(size_t)s * kMmaCols + g];
+        for (int g = 0; g < G; ++g) gain += w[(size_t)s * kMmaCols + g] * s_inv[g];
         const float sn = fmaf(alpha, s_old[s], gain);
         Su[s] = sn;
         const int ps = s_pos[s];
@@ -605,7 +613,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
 
     // ---- (v) eviction and in-place insert, (vi) length ------------------------------------------
     float s_new = 0.f;
-    for (int g = 0; g < G; ++g) s_new += w[(size_t)cnt * kMmaCols + g];
+    for (int g = 0; g < G; ++g) s_new += w[(size_t)cnt * kMmaCols + g] * s_inv[g];
     if (tid == 0) {
         int target = full ? -2 : cnt;
         if (full) {
