@@ -648,16 +648,30 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     }
 }
 
+// The dynamic shared-memory limit of a kernel is raised once per device and size, not per launch
+// (the call is a driver round trip).  The kernel is a template argument so that every kernel has
+// its own record.
+template <auto Kern>
+cudaError_t allow_dynamic_smem(size_t smem)
+{
+    static size_t granted[kMaxDevices] = {};
+    if (smem <= 48 * 1024) return cudaSuccess;
+    const int dev = current_device_index();
+    if (smem > granted[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        granted[dev] = smem;
+    }
+    return cudaSuccess;
+}
+
 template <typename T, int D>
 cudaError_t launch_group_mma(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
                              const void *v_new, void *out, int32_t *evicted, cudaStream_t s)
 {
     const size_t smem = group_mma_smem_bytes(c.M, D);
     auto kern = decode_step_group_mma_kernel<T, D>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    if (cudaError_t e = allow_dynamic_smem<decode_step_group_mma_kernel<T, D>>(smem); e != cudaSuccess) return e;
     kern<<<c.U, kGroupThreads, smem, s>>>(c, G, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
                                            static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
     count_launch();
@@ -671,10 +685,7 @@ cudaError_t launch_group_n(const CacheView &c, int G, float alpha, const void *q
     const size_t smem = decode_group_smem_bytes(c.M, G, D);
     if (smem > 220 * 1024) return cudaErrorInvalidValue;
     auto kern = decode_step_group_kernel<T, D, GMAX>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    if (cudaError_t e = allow_dynamic_smem<decode_step_group_kernel<T, D, GMAX>>(smem); e != cudaSuccess) return e;
     kern<<<c.U, kGroupThreads, smem, s>>>(c, G, alpha, static_cast<const T *>(q), static_cast<const T *>(k_new),
                                            static_cast<const T *>(v_new), static_cast<T *>(out), evicted);
     count_launch();
