@@ -570,21 +570,29 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
             for (int i = 0; i < VL; ++i) vcur[x][i] = vnxt[x][i];
     }
     // oacc[t]: (element E*r + t, queries 2c, 2c+1), (element E*r + E/2 + t, queries 2c, 2c+1)
-#pragma unroll
-    for (int t = 0; t < MT; ++t) {
+    // Within its E elements of a row a lane's values are stored rotated by rot(r, c), so that the 32
+    // lanes of one store hit 32 banks (unrotated, they would share two); the reader undoes it.
+    {
+        const int rot = 4 * (r / (32 / E)) + cq;
         float *pw = part + (size_t)warp * kMmaCols * D;
-        pw[(2 * cq) * D + E * r + t] = oacc[t][0];
-        pw[(2 * cq + 1) * D + E * r + t] = oacc[t][1];
-        pw[(2 * cq) * D + E * r + E / 2 + t] = oacc[t][2];
-        pw[(2 * cq + 1) * D + E * r + E / 2 + t] = oacc[t][3];
+#pragma unroll
+        for (int t = 0; t < MT; ++t) {
+            const int lo = E * r + ((t + rot) % E), hi = E * r + ((E / 2 + t + rot) % E);
+            pw[(2 * cq) * D + lo] = oacc[t][0];
+            pw[(2 * cq + 1) * D + lo] = oacc[t][1];
+            pw[(2 * cq) * D + hi] = oacc[t][2];
+            pw[(2 * cq + 1) * D + hi] = oacc[t][3];
+        }
     }
     cp_async_wait_all();                       // this thread's staged scores and positions
     __syncthreads();
     for (int x = tid; x < G * D; x += kGroupThreads) {
+        const int g = x / D, d = x % D, row = d / E;
+        const int col = g * D + E * row + ((d % E + 4 * (row / (32 / E)) + (g >> 1)) % E);
         float o = 0.f;
 #pragma unroll
-        for (int wv = 0; wv < NW; ++wv) o += part[(size_t)wv * kMmaCols * D + x];
-        out[(size_t)u * G * D + x] = Elem<T>::from_float(o * s_inv[x / D]);
+        for (int wv = 0; wv < NW; ++wv) o += part[(size_t)wv * kMmaCols * D + col];
+        out[(size_t)u * G * D + x] = Elem<T>::from_float(o * s_inv[g]);
     }
 
     // ---- (iv) S <- alpha*S + sum_g a_g ; candidates for eviction ---------------------------------
