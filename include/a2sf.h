@@ -125,6 +125,14 @@ int a2sf_rescore(const a2sf_params *p, int32_t n,
                  const float *lse, float *scores, int32_t *kept_idx,
                  void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* Selection alone (Sec. 3.1, Sec. 4.1): kept_idx from a given score vector, exactly the last
+ * step of a2sf_prefill / a2sf_rescore -- every position >= n-R plus, of the others, all but the
+ * n-M lowest under (score, position) ascending.  scores [B][H][n] fp32 (input, non-negative),
+ * kept_idx [B][H][min(n,M)] int32 (output, ascending).  Lets a caller re-select under another
+ * budget or recent window without recomputing scores. */
+int a2sf_select(const a2sf_params *p, int32_t n, const float *scores, int32_t *kept_idx,
+                void *cuda_stream);
+
 /* Per-head forgetting factors (the paper's Limitation section suggests a distinct factor per
  * layer and head instead of one uniform value).  `alphas` is a DEVICE array [B][H] fp32, one
  * factor per unit; p->alpha is ignored.  Values outside [0, 1] (or NaN) cannot be rejected on
@@ -150,9 +158,10 @@ int a2sf_rescore_per_head(const a2sf_params *p, int32_t n,
  * and the call returns after the stream has drained.  The device copies of k, v,
  * scores and kept_idx stay valid in the workspace for a2sf_cache_load: their
  * addresses are returned through dev_k, dev_v, dev_scores, dev_kept (any may be NULL).
- * With two or more batch rows the work is pipelined over chunks of rows on two streams that
- * the call creates and destroys: they start after what is already queued on cuda_stream,
- * and cuda_stream (and the call) continues only when they have drained. */
+ * With two or more batch rows the work is pipelined over chunks of rows on two internal
+ * streams (created once per device on first use and kept): they start after what is already
+ * queued on cuda_stream, and cuda_stream (and the call) continues only when they have drained.
+ * Chunked calls on one device are serialised against each other. */
 size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n);
 
 int a2sf_prefill_host(const a2sf_params *p, int32_t n,
@@ -165,10 +174,11 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n,
 /* Prefill without any allocation, for callers that cannot call cudaMalloc (an
  * engine whose own allocator owns the device, a plugin that only sees one layer's
  * tensors, a loop that must not hit an allocation's implicit synchronisation).
- * The paper has no counterpart: this is the same computation as a2sf_prefill, run
- * by the CUDA-core kernels, with the per-row log-sum-exp scratch held in a fixed
- * 4 MiB array inside the library's device image (every GPU that loads the library
- * carries it until the process exits).
+ * The paper has no counterpart: this is the same computation as a2sf_prefill, with
+ * the per-row log-sum-exp scratch held in a fixed 4 MiB array inside the library's
+ * device image (every GPU that loads the library carries it until the process
+ * exits).  It runs the same kernels as a2sf_prefill except that, having no workspace
+ * for an fp16 copy of V, bf16 storage multiplies P V with two bf16 terms.
  *   - Limit: B*H*n <= a2sf_prefill_static_scratch_max_rows() (1,048,576); larger
  *     calls return A2SF_ERR_WORKSPACE and launch nothing.
  *   - The first call on each device looks up the array's device address (a short
@@ -352,6 +362,22 @@ int64_t a2sf_kernel_launch_count(void);
  * status is set the tensor-core prefill kernels return without working, so results
  * of calls made after a timeout and before this call are undefined. */
 int a2sf_last_device_status(void *cuda_stream);
+
+/* Self-test of the device-side failure path (the paper has no counterpart; a test hook, not
+ * part of the method).  Every wait inside the kernels of this library is bounded: a wait that
+ * runs out poisons its CTA, the kernel unwinds and raises the sticky status that
+ * a2sf_last_device_status reports.  This call exercises exactly that, harmlessly: it launches one
+ * CTA whose first thread waits -- through the library's own bounded wait, with `limit_cycles`
+ * SM clocks as the limit -- on a barrier at which nobody ever arrives, then raises the status
+ * word of the tensor-core prefill kernels (which = 0) or of the generation-step kernels
+ * (which = 1).  Nothing traps and nothing waits without a bound.
+ *   report : DEVICE int64[4], written by the kernel: [0] 1 if the wait reported failure,
+ *            [1] SM clocks the wait took, [2] SM clocks of a second wait in the same CTA (it
+ *            returns at once because the CTA is poisoned), [3] 1 if that second wait failed too.
+ *   limit_cycles in [1, A2SF_SELFTEST_MAX_WAIT_CYCLES]; INVALID_ARG otherwise.
+ * Afterwards a2sf_last_device_status returns A2SF_ERR_TIMEOUT once, then A2SF_OK. */
+#define A2SF_SELFTEST_MAX_WAIT_CYCLES 2000000000ll
+int a2sf_selftest_bounded_wait(int32_t which, int64_t limit_cycles, int64_t *report, void *cuda_stream);
 
 const char *a2sf_status_string(int status);
 

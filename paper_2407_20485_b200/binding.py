@@ -78,6 +78,8 @@ def _load():
         "a2sf_cache_import": (ctypes.c_int, [vp] * 8),
         "a2sf_kernel_launch_count": (ctypes.c_int64, []),
         "a2sf_last_device_status": (ctypes.c_int, [vp]),
+        "a2sf_select": (ctypes.c_int, [ctypes.POINTER(a2sf_params), ctypes.c_int32, vp, vp, vp]),
+        "a2sf_selftest_bounded_wait": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int64, vp, vp]),
         "a2sf_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     }
     for name, (res, args) in sigs.items():
@@ -130,6 +132,24 @@ def a2sf_kernel_launch_count() -> int:
 
 def a2sf_last_device_status(stream=None) -> int:
     return int(lib.a2sf_last_device_status(_stream(stream)))
+
+
+def a2sf_select(p: a2sf_params, scores: torch.Tensor, kept_idx=None, stream=None) -> torch.Tensor:
+    """Selection alone: the kept set of ``scores`` [B, H, n] (fp32, contiguous)."""
+    assert scores.dtype == torch.float32 and scores.is_contiguous() and scores.dim() == 3
+    n = scores.shape[2]
+    if kept_idx is None:
+        kept_idx = torch.empty((p.B, p.H, min(n, p.budget)), dtype=torch.int32, device=scores.device)
+    _check(lib.a2sf_select(ctypes.byref(p), n, _ptr(scores), _ptr(kept_idx), _stream(stream)), "a2sf_select")
+    return kept_idx
+
+
+def a2sf_selftest_bounded_wait(which: int, limit_cycles: int, stream=None) -> torch.Tensor:
+    """Runs the bounded-wait self-test; returns the kernel's report (int64[4], on the device)."""
+    report = torch.zeros((4,), dtype=torch.int64, device="cuda")
+    _check(lib.a2sf_selftest_bounded_wait(which, limit_cycles, report.data_ptr(), _stream(stream)),
+           "a2sf_selftest_bounded_wait")
+    return report
 
 
 def a2sf_prefill_workspace_bytes(p: a2sf_params, n: int) -> int:

@@ -3,6 +3,7 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "common.cuh"
@@ -16,7 +17,7 @@ static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a
 static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 static inline int elem_bytes(int dtype) { return dtype == A2SF_F32 ? 4 : 2; }
 
-static int check_params(const a2sf_params *p)
+int check_params(const a2sf_params *p)
 {
     if (!p) return A2SF_ERR_INVALID_ARG;
     if (p->B < 1 || p->H < 1 || p->budget < 1 || p->recent < 0 || p->recent > p->budget)
@@ -33,12 +34,12 @@ static int check_params(const a2sf_params *p)
     return A2SF_OK;
 }
 
-static inline float eff_scale(const a2sf_params *p)
+float eff_scale(const a2sf_params *p)
 {
     return p->scale > 0.f ? p->scale : 1.0f / std::sqrt((float)p->d);
 }
 
-static int check_strides(const a2sf_params *p, int64_t sb, int64_t sh, int64_t st)
+int check_strides(const a2sf_params *p, int64_t sb, int64_t sh, int64_t st)
 {
     const int vec = 16 / elem_bytes(p->dtype);
     if (st < p->d || sh < 1 || sb < 1) return A2SF_ERR_INVALID_ARG;
@@ -62,6 +63,32 @@ static int run_scores_and_select(const a2sf_params *p, int n, PrefillArgs &a, in
     if (launch_select(a.scores, kept, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
         return A2SF_ERR_CUDA;
     return A2SF_OK;
+}
+
+// Two side streams and the events that fork from / join into the caller's stream, for the
+// chunked host-buffer prefill.  Built once per device, on first use, and kept for the life of
+// the process (creating and destroying them on every call costs several driver round trips).
+struct HostPipeline {
+    cudaStream_t side[2] = {nullptr, nullptr};
+    cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
+    bool ok = false;
+    std::mutex mu;          // one chunked call at a time per device: the calls share the streams
+};
+
+static HostPipeline *host_pipeline()
+{
+    static std::once_flag once[kMaxDevices];
+    static HostPipeline pipes[kMaxDevices];
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
+        HostPipeline &hp = pipes[dev];
+        bool ok = cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess;
+        for (int x = 0; ok && x < 2; ++x)
+            ok = cudaStreamCreateWithFlags(&hp.side[x], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.done[x], cudaEventDisableTiming) == cudaSuccess;
+        hp.ok = ok;
+    });
+    return &pipes[dev];
 }
 
 }  // namespace a2sf
@@ -256,6 +283,17 @@ int a2sf_rescore_per_head(const a2sf_params *p, int32_t n, const void *q, const 
                         workspace, workspace_bytes, cuda_stream);
 }
 
+int a2sf_select(const a2sf_params *p, int32_t n, const float *scores, int32_t *kept_idx, void *cuda_stream)
+{
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (n < 1 || !scores || !kept_idx || !aligned(scores, 4) || !aligned(kept_idx, 4)) return A2SF_ERR_INVALID_ARG;
+    if (launch_select(scores, kept_idx, p->B * p->H, n, p->budget, p->recent,
+                      static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
 size_t a2sf_prefill_host_workspace_bytes(const a2sf_params *p, int32_t n)
 {
     if (check_params(p) != A2SF_OK || n < 1) return 0;
@@ -307,14 +345,13 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const
             return A2SF_ERR_CUDA;
         if (cudaStreamSynchronize(s) != cudaSuccess) return A2SF_ERR_CUDA;
     } else {
-        cudaStream_t side[2] = {nullptr, nullptr};
-        cudaEvent_t start = nullptr, done[2] = {nullptr, nullptr};
-        bool ok = cudaEventCreateWithFlags(&start, cudaEventDisableTiming) == cudaSuccess;
-        for (int x = 0; ok && x < 2; ++x)
-            ok = cudaStreamCreateWithFlags(&side[x], cudaStreamNonBlocking) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&done[x], cudaEventDisableTiming) == cudaSuccess;
+        HostPipeline *hp = host_pipeline();
+        if (!hp->ok) return A2SF_ERR_CUDA;
+        std::lock_guard<std::mutex> pipeline_lock(hp->mu);
+        cudaStream_t *side = hp->side;
+        cudaEvent_t start = hp->start, *done = hp->done;
         // work already queued on the caller's stream comes first
-        ok = ok && cudaEventRecord(start, s) == cudaSuccess;
+        bool ok = cudaEventRecord(start, s) == cudaSuccess;
         for (int x = 0; ok && x < 2; ++x) ok = cudaStreamWaitEvent(side[x], start, 0) == cudaSuccess;
         const size_t eb = elem_bytes(p->dtype);
         const int rows_per = (p->B + chunks - 1) / chunks;
@@ -344,14 +381,11 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const
         }
         // the caller's stream continues only after both side streams have drained
         for (int x = 0; x < 2; ++x)
-            if (side[x] && done[x] && cudaEventRecord(done[x], side[x]) == cudaSuccess)
-                cudaStreamWaitEvent(s, done[x], 0);
+            if (cudaEventRecord(done[x], side[x]) != cudaSuccess || cudaStreamWaitEvent(s, done[x], 0) != cudaSuccess)
+                ok = false;
         const bool drained = cudaStreamSynchronize(s) == cudaSuccess;
-        for (int x = 0; x < 2; ++x) {
-            if (side[x]) { cudaStreamSynchronize(side[x]); cudaStreamDestroy(side[x]); }
-            if (done[x]) cudaEventDestroy(done[x]);
-        }
-        if (start) cudaEventDestroy(start);
+        if (!ok)                                   // a failed fork or join: leave nothing running behind
+            for (int x = 0; x < 2; ++x) cudaStreamSynchronize(side[x]);
         if (rc2 != A2SF_OK) return rc2;
         if (!ok || !drained) return A2SF_ERR_CUDA;
     }
@@ -696,6 +730,19 @@ int a2sf_last_device_status(void *cuda_stream)
     const int a = read_and_clear_tc_status(static_cast<cudaStream_t>(cuda_stream));
     const int b = read_and_clear_decode_status(static_cast<cudaStream_t>(cuda_stream));
     return a != A2SF_OK ? a : b;
+}
+
+int a2sf_selftest_bounded_wait(int32_t which, int64_t limit_cycles, int64_t *report, void *cuda_stream)
+{
+    if ((which != 0 && which != 1) || !report || !aligned(report, 8)) return A2SF_ERR_INVALID_ARG;
+    if (limit_cycles < 1 || limit_cycles > A2SF_SELFTEST_MAX_WAIT_CYCLES) return A2SF_ERR_INVALID_ARG;
+    int *word = which == 0 ? tc_status_word() : decode_status_word();
+    if (!word) return A2SF_ERR_CUDA;
+    static_assert(sizeof(long long) == sizeof(int64_t), "report words");
+    if (launch_wait_probe(word, (long long)limit_cycles, reinterpret_cast<long long *>(report),
+                          static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    return A2SF_OK;
 }
 
 const char *a2sf_status_string(int status)

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/a2sf.h"
 
 namespace a2sf {
@@ -60,12 +62,23 @@ template <> struct Elem<__half> {
     __device__ static __half from_float(float x) { return __float2half_rn(x); }
 };
 
-// streaming 16-byte load that does not displace L1 lines
+// streaming 16-byte load that does not displace L1 lines; only for data that no thread writes
+// while the kernel runs (the non-coherent path)
 __device__ __forceinline__ uint4 ld_stream16(const void *p)
 {
     uint4 r;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+
+// the same for rows that the kernel itself may overwrite later in the launch (a cache row that
+// the new token replaces): the ordinary coherent path, still without an L1 allocation
+__device__ __forceinline__ uint4 ld_stream16_rw(const void *p)
+{
+    uint4 r;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
     return r;
 }
 
@@ -106,6 +119,42 @@ inline int current_device_index()
     return d;
 }
 
+// Number of SMs of the current device, looked up once per device.
+inline int device_sm_count()
+{
+    static std::once_flag once[kMaxDevices];
+    static int count[kMaxDevices] = {};
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
+        if (cudaDeviceGetAttribute(&count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) count[dev] = 0;
+    });
+    return count[dev];
+}
+
+// The dynamic shared-memory limit of a kernel is raised once per device and size, not per launch
+// (the call is a driver round trip), under a lock.  The kernel is a template argument so that
+// every kernel has its own record.
+template <auto Kern>
+cudaError_t allow_dynamic_smem(size_t smem)
+{
+    static std::mutex mu;
+    static size_t granted[kMaxDevices] = {};
+    if (smem <= 48 * 1024) return cudaSuccess;
+    const int dev = current_device_index();
+    std::lock_guard<std::mutex> lock(mu);
+    if (smem > granted[dev]) {
+        const cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        granted[dev] = smem;
+    }
+    return cudaSuccess;
+}
+
+// ---- host-side argument checks shared by every entry point (api.cu) ----------------------
+int check_params(const a2sf_params *p);                                    // shape, policy, dtype, flags
+int check_strides(const a2sf_params *p, int64_t sb, int64_t sh, int64_t st);   // element strides of q/k/v/out
+float eff_scale(const a2sf_params *p);                                     // scale, or 1/sqrt(d) when 0
+
 // ---- kernel launchers (one per translation unit) -----------------------------
 struct PrefillArgs {
     const void *q, *k, *v;
@@ -134,6 +183,7 @@ size_t prefill_tc_extra_bytes(int dtype, size_t units, int n, int d);
 cudaError_t launch_prefill_pass1_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_t s);
 int read_and_clear_tc_status(cudaStream_t s);
+int *tc_status_word();       // device address of that status word on the current device (nullptr on failure)
 
 cudaError_t launch_select(const float *scores, int32_t *kept, int U, int n, int M, int R,
                           cudaStream_t s);
@@ -174,6 +224,8 @@ __device__ __forceinline__ float unit_alpha(const float *alpha_vec, int u, float
 }
 
 int read_and_clear_decode_status(cudaStream_t s);
+int *decode_status_word();   // device address of that status word on the current device (nullptr on failure)
+cudaError_t launch_wait_probe(int *status_word, long long limit_cycles, long long *report, cudaStream_t s);
 
 // grouped query heads (G query heads per K/V head)
 cudaError_t launch_group_sum(const float *per_head, float *out, int G, int n, size_t units, cudaStream_t s);

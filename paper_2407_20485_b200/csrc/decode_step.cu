@@ -19,17 +19,6 @@ static __device__ int g_decode_status = 0;
 
 namespace {
 
-int *decode_status_word()
-{
-    static int *ptr[kMaxDevices] = {};
-    const int dev = current_device_index();
-    if (!ptr[dev]) {
-        void *p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_decode_status) == cudaSuccess) ptr[dev] = static_cast<int *>(p);
-    }
-    return ptr[dev];
-}
-
 constexpr int kDecodeThreads = 256;
 constexpr int kSplitMinBudget = 512;         // split-K only pays for long caches
 
@@ -168,7 +157,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         for (int x = 0; x < kU; ++x) {
             const int row = ((bidx * kU + x) * NW + warp) * RPW + rsel;
             r[x] = make_uint4(0, 0, 0, 0);
-            if (bidx < nb && row < nloc) r[x] = ld_stream16(base + (size_t)(s0 + row) * D + sub * VEC);
+            if (bidx < nb && row < nloc) r[x] = ld_stream16_rw(base + (size_t)(s0 + row) * D + sub * VEC);
         }
     };
     // batch index b: K batch b for b < nb, V batch b - nb after that
@@ -451,6 +440,7 @@ struct StreamShared {
     float red[kStreamConsumerWarps];
     int target;
     int abort_flag;
+    int unit_ok;        // 0 when a wait of the current unit ran out (one decision for all consumers)
 };
 
 template <typename T, int D>
@@ -668,7 +658,12 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             if (rsel == 0)
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) part[warp * D + sub * VEC + e] = acc[e];
+            // All of this unit's waits lie behind.  If one of them ran out, its rows are not
+            // trustworthy: the unit's cached state (scores, rows, counters) is then left as it
+            // was.  One thread decides for all, so the state is never half updated.
+            if (tid == 0) sh->unit_ok = !*abort_flag;
             consumer_barrier();
+            const bool alive = sh->unit_ok != 0;
             if (tid < D) {
                 float o = 0.f;
 #pragma unroll
@@ -691,7 +686,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                 else if (x_pre == 1) { s_old = s_pre[1]; ps = pos_pre[1]; }
                 else { s_old = Su[s_]; ps = posu[s_]; }
                 const float sn = fmaf(alpha, s_old, a);
-                Su[s_] = sn;
+                if (alive) Su[s_] = sn;
                 if (full && ps <= newest_evictable) {
                     const unsigned long long key =
                         ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
@@ -714,7 +709,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             consumer_barrier();
 
             const int target = sh->target;
-            if (target >= 0) {
+            if (target >= 0 && alive) {
                 if (tid < LPR)
                     *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
                         *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
@@ -722,7 +717,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                     *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
                         *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
             }
-            if (tid == 0 && !*abort_flag) {
+            if (tid == 0 && alive) {
                 if (target >= 0) {
                     Su[target] = a_self;
                     posu[target] = p;
@@ -756,11 +751,7 @@ cudaError_t launch_split(const CacheView &c, int cluster_size, float alpha, cons
     const size_t per_max = ((size_t)c.M + cluster_size - 1) / cluster_size;
     const size_t smem = ((per_max + 1 + 3) & ~(size_t)3) * 4 + (size_t)(NT / 32) * D * 4 + (NT / 32) * 4;
     auto kern = decode_step_split_kernel<T, D, NT>;
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
-        if (e != cudaSuccess) return e;
-    }
+    if (cudaError_t e = allow_dynamic_smem<decode_step_split_kernel<T, D, NT>>(smem); e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)c.U * cluster_size);
     cfg.blockDim = dim3(NT);
@@ -795,23 +786,15 @@ cudaError_t launch_stream(const CacheView &c, float alpha, const float *alpha_ve
     if (stages > kMaxStreamStages) stages = kMaxStreamStages;
     const size_t smem = fixed + (size_t)stages * kChunkBytes;
     auto kern = decode_step_stream_kernel<T, D>;
-    static int sm_count[kMaxDevices] = {};
-    const int dev = current_device_index();
-    if (sm_count[dev] == 0) cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
-    const int num_sms = sm_count[dev];
+    const int num_sms = device_sm_count();
+    if (num_sms <= 0) return cudaErrorUnknown;
     // Few units with long caches would leave most SMs idle: split each unit over a cluster.
     if (c.M >= kSplitMinBudget && c.U * 2 <= num_sms) {
         int cs = 2;
         while (cs < 8 && c.U * cs * 2 <= 2 * num_sms) cs *= 2;
         return launch_split<T, D>(c, cs, alpha, alpha_vec, q, k_new, v_new, out, evicted, s);
     }
-    static cudaError_t attr_err[kMaxDevices] = {};
-    static size_t attr_smem[kMaxDevices] = {};
-    if (smem > attr_smem[dev]) {
-        attr_err[dev] = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attr_smem[dev] = smem;
-    }
-    if (attr_err[dev] != cudaSuccess) return attr_err[dev];
+    if (cudaError_t e = allow_dynamic_smem<decode_step_stream_kernel<T, D>>(smem); e != cudaSuccess) return e;
     int *status = decode_status_word();
     if (!status) return cudaErrorUnknown;
     const int grid = c.U < ctas_per_sm * num_sms ? c.U : ctas_per_sm * num_sms;
@@ -837,6 +820,19 @@ cudaError_t launch_decode_step(const CacheView &c, float alpha, const float *alp
     default: return A2SF_DISPATCH(__half);
     }
 #undef A2SF_DISPATCH
+}
+
+// device address of the status word, looked up once per device
+int *decode_status_word()
+{
+    static std::once_flag once[kMaxDevices];
+    static int *ptr[kMaxDevices] = {};
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_decode_status) == cudaSuccess) ptr[dev] = static_cast<int *>(p);
+    });
+    return ptr[dev];
 }
 
 int read_and_clear_decode_status(cudaStream_t s)

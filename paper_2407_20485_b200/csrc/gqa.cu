@@ -656,23 +656,6 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     }
 }
 
-// The dynamic shared-memory limit of a kernel is raised once per device and size, not per launch
-// (the call is a driver round trip).  The kernel is a template argument so that every kernel has
-// its own record.
-template <auto Kern>
-cudaError_t allow_dynamic_smem(size_t smem)
-{
-    static size_t granted[kMaxDevices] = {};
-    if (smem <= 48 * 1024) return cudaSuccess;
-    const int dev = current_device_index();
-    if (smem > granted[dev]) {
-        const cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        granted[dev] = smem;
-    }
-    return cudaSuccess;
-}
-
 template <typename T, int D>
 cudaError_t launch_group_mma(const CacheView &c, int G, float alpha, const void *q, const void *k_new,
                              const void *v_new, void *out, int32_t *evicted, cudaStream_t s)

@@ -20,7 +20,6 @@ static __device__ __align__(256) float g_static_lse[kStaticLseFloats];
 
 namespace {
 
-constexpr int kMaxDevices = 64;
 std::mutex g_mu;
 float *g_lse_addr[kMaxDevices] = {};
 
@@ -55,23 +54,19 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
                                            int64_t stride_h, int64_t stride_t, void *out,
                                            float *scores, int32_t *kept_idx, void *cuda_stream)
 {
-    if (!p || n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
-    if (p->B < 1 || p->H < 1 || p->budget < 1 || p->recent < 0 || p->recent > p->budget ||
-        !(p->alpha >= 0.f && p->alpha <= 1.f) || !(p->scale >= 0.f) || isinf(p->scale))
-        return A2SF_ERR_INVALID_ARG;
-    if ((p->dtype != A2SF_F32 && p->dtype != A2SF_BF16 && p->dtype != A2SF_F16) ||
-        (p->d != 64 && p->d != 128))
-        return A2SF_ERR_UNSUPPORTED;
-    const int vec = p->dtype == A2SF_F32 ? 4 : 8;
-    if (stride_t < p->d || stride_h < 1 || stride_b < 1 || stride_t % vec || stride_h % vec ||
-        stride_b % vec || !aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+    // the same checks, in the same order, as a2sf_prefill
+    int rc = check_params(p);
+    if (rc != A2SF_OK) return rc;
+    if (n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
+    if ((rc = check_strides(p, stride_b, stride_h, stride_t)) != A2SF_OK) return rc;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(scores) & 3) || (reinterpret_cast<uintptr_t>(kept_idx) & 3))
         return A2SF_ERR_INVALID_ARG;
     // the scratch is fixed: refuse what does not fit rather than overrun it
     if ((size_t)p->B * (size_t)p->H * (size_t)n > kStaticLseFloats) return A2SF_ERR_WORKSPACE;
 
     float *lse = nullptr;
-    const int rc = static_lse_address(&lse);
-    if (rc != A2SF_OK) return rc;
+    if ((rc = static_lse_address(&lse)) != A2SF_OK) return rc;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     PrefillArgs a;
@@ -81,15 +76,20 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
     a.st = Strides{stride_b, stride_h, stride_t};
     a.st_kv = a.st; a.G = 1;
     a.B = p->B; a.H = p->H; a.n = n; a.d = p->d;
-    a.scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf((float)p->d);
+    a.scale = eff_scale(p);
     a.alpha = p->alpha;
     a.alpha_vec = nullptr;
-    a.skip_zero_rows = 0;
-    a.window_rows = 0;
+    a.skip_zero_rows = (p->flags & A2SF_FLAG_SKIP_ZERO_WEIGHT_ROWS) ? 1 : 0;
+    a.window_rows = p->score_window;
+    // no workspace, hence no fp16 copy of V: 16-bit storage with d = 128 still runs on the tensor
+    // cores (bf16 multiplies P as two bf16 terms with V as it is), everything else on CUDA cores
     a.v_half = nullptr;
     a.v_flag = nullptr;
-    if (launch_prefill_pass1_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
-    if (launch_prefill_pass2_simt(p->dtype, a, s) != cudaSuccess) return A2SF_ERR_CUDA;
+    const bool tc = prefill_tc_supported(p->dtype, a);
+    if ((tc ? launch_prefill_pass1_tc(p->dtype, a, s) : launch_prefill_pass1_simt(p->dtype, a, s)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
+    if ((tc ? launch_prefill_pass2_tc(p->dtype, a, s) : launch_prefill_pass2_simt(p->dtype, a, s)) != cudaSuccess)
+        return A2SF_ERR_CUDA;
     if (launch_select(scores, kept_idx, p->B * p->H, n, p->budget, p->recent, s) != cudaSuccess)
         return A2SF_ERR_CUDA;
     return A2SF_OK;

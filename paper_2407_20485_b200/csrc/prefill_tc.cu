@@ -954,6 +954,18 @@ cudaError_t launch_prefill_pass2_tc(int dtype, const PrefillArgs &a, cudaStream_
     return cudaGetLastError();
 }
 
+int *tc_status_word()
+{
+    static std::once_flag once[kMaxDevices];
+    static int *ptr[kMaxDevices] = {};
+    const int dev = current_device_index();
+    std::call_once(once[dev], [dev] {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_tc_status) == cudaSuccess) ptr[dev] = static_cast<int *>(p);
+    });
+    return ptr[dev];
+}
+
 int read_and_clear_tc_status(cudaStream_t s)
 {
     int v = 0, zero = 0;

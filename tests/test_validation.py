@@ -82,5 +82,12 @@ def test_null_cache_and_size_queries():
     assert lib.a2sf_ideal_similarity_workspace_bytes(ctypes.byref(p), 32769) == 0
     assert lib.a2sf_ideal_similarity_workspace_bytes(ctypes.byref(p), 1024) >= 2 * 1024 * 16
     assert lib.a2sf_prefill_static_scratch_max_rows() == 1 << 20
+    assert lib.a2sf_select(ctypes.byref(p), 0, FAKE, FAKE, None) == INVALID
+    assert lib.a2sf_select(ctypes.byref(p), 64, None, FAKE, None) == INVALID
+    assert lib.a2sf_select(ctypes.byref(_p(budget=0)), 64, FAKE, FAKE, None) == INVALID
+    # the bounded-wait self-test refuses anything that is not a short, bounded wait before any CUDA call
+    for which, limit, rep in ((2, 1000, FAKE), (-1, 1000, FAKE), (0, 0, FAKE), (0, 2_000_000_001, FAKE),
+                              (1, 1000, None), (1, 1000, ctypes.c_void_p(0x1004))):
+        assert lib.a2sf_selftest_bounded_wait(which, limit, rep, None) == INVALID
     for code in (0, -1, -2, -3, -4, -5, 99):
         assert len(lib.a2sf_status_string(code)) > 0
