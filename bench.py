@@ -34,9 +34,31 @@ METRIC = "a2sf_decode_step_hbm_gbps"
 UNIT = "GB/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 NOMINAL = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode_step_stream_kernel launch (ncu, config 4;
-# the capture is summarised in profiles/launch_list_llama2_13b.md).  Set to None when the kernel changes.
-NCU_DECODE_TRAFFIC = {("llama2_13b", 32): 342910000}
+# The ncu DRAM traffic of one decode launch is kept as a data line beside the launch-list summary,
+# together with a hash of the kernel's sources at the time of the capture.
+TRAFFIC_RECORD = ROOT / "profiles" / "launch_list_llama2_13b.md"
+
+
+def ncu_decode_traffic(workload: str, batch: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one decode_step_stream_kernel launch from
+    the committed ncu capture -- or None when there is no capture of this workload, or when any
+    source of the kernel has changed since it was taken (a stale figure is not a measurement)."""
+    import hashlib
+
+    try:
+        for line in TRAFFIC_RECORD.read_text().splitlines():
+            if not line.startswith("bench-data:"):
+                continue
+            rec = json.loads(line[len("bench-data:"):])
+            if rec.get("workload") != workload or rec.get("batch") != batch:
+                continue
+            for rel, digest in rec["sources"].items():
+                if hashlib.sha256((ROOT / rel).read_bytes()).hexdigest() != digest:
+                    return None
+            return int(rec["dram_bytes_per_launch"])
+    except (OSError, ValueError, KeyError):
+        pass
+    return None
 
 
 def load_peaks():
@@ -215,9 +237,15 @@ def run_ours(args):
     for _ in range(reps_r):       # the whole prefill under the same (short-run) clocks
         a2sf.a2sf_prefill(p, q, k, v, out=out, scores=scores, kept_idx=kept, lse=lse, workspace=ws)
     er[2].record()
+    es_ = cuda_events(2)
+    es_[0].record()
+    for _ in range(reps_r):       # the selection (K3) alone, from the scores just written
+        a2sf.a2sf_select(p, scores, kept_idx=kept)
+    es_[1].record()
     torch.cuda.synchronize()
     rescore_ms = er[0].elapsed_time(er[1]) / reps_r
     prefill_short_ms = er[1].elapsed_time(er[2]) / reps_r
+    select_ms = es_[0].elapsed_time(es_[1]) / reps_r
 
     # ---- separate line: the scoring pass without the rows whose forgetting weight is exactly
     # zero in fp32 (bit-identical scores, less work; NOT part of the headline step above)
@@ -340,17 +368,23 @@ def run_ours(args):
                     "frac_of_nominal_bf16": prefill_tflops / scale_units / NOMINAL["bf16_tflops"],
                     "passes": {
                         "scores_and_selection_ms": rescore_ms,
-                        "scores_tflops": U * flops["pass2"] / (rescore_ms * 1e-3) / 1e12,
+                        "scores_ms": rescore_ms - select_ms,
+                        "selection_ms": select_ms,
+                        "scores_tflops": U * flops["pass2"] / ((rescore_ms - select_ms) * 1e-3) / 1e12,
                         "prefill_ms": prefill_short_ms,
                         "attention_ms": prefill_short_ms - rescore_ms,
                         "attention_tflops": U * flops["pass1"] / ((prefill_short_ms - rescore_ms) * 1e-3) / 1e12,
                         "note": "this rank, 5 back-to-back repetitions after the timed region (shorter "
-                                "run, higher clocks than inside it); attention = prefill - (scores + "
-                                "selection), includes the fp16 copy of V for bf16 storage"}},
+                                "run, higher clocks than inside it); K1 attention = prefill - (scores + "
+                                "selection), includes the fp16 copy of V for bf16 storage; K2 scores = "
+                                "a2sf_rescore - a2sf_select; K3 selection = a2sf_select; K4 = "
+                                "phases_ms_per_step.cache_load"},
+                    "roofline": prefill_roofline(w, U, prefill_tflops / scale_units, max_prefill_ms / K, peaks,
+                                                 clocks.get("sm_mhz"))},
         "roofline": {"kernel": "decode_step_stream_kernel", "bound": "hbm", "achieved": achieved,
                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8TBps": achieved / NOMINAL["hbm_gbs"],
-                     "traffic": NCU_DECODE_TRAFFIC.get((w.name, w.B)), "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
+                     "traffic": ncu_decode_traffic(w.name, w.B), "bytes_per_launch": bytes_per_launch, "launch_us": launch_us},
         "prefill_zero_weight_rows_skipped": windowed,
         "prefill_streamed_row_by_row": streamed,
         "gpu_launches": int(launches),
@@ -380,6 +414,29 @@ def run_ours(args):
     if rank == 0:
         print(json.dumps(result))
     a2dist.finalize()
+
+
+def prefill_roofline(w, U, tflops, ms, peaks, sm_mhz):
+    """The prefill against its two ceilings.  Tensor: the causal flops at the measured sustained
+    and the nominal dense bf16 rate.  Special-function unit: the two passes evaluate one exp2 per
+    logit of every 128x128 tile they touch (diagonal tiles in full), and an SM retires 16 of them
+    per clock (measured: 15.8 per clock with the multiply-add and add of the scoring loop around
+    them).  The kernels overlap the two only partly, so the time is compared with each and with
+    their sum."""
+    T = (w.n + 127) // 128
+    tiles = U * T * (T + 1) // 2
+    exps = 2 * tiles * 128 * 128
+    mhz = sm_mhz or 1800.0
+    sfu_ms = exps / (16.0 * 148 * mhz * 1e6) * 1e3
+    fl = w.prefill_flops_per_unit()
+    tensor_ms = U * (fl["pass1"] + fl["pass2"]) / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+    return {"bound": "tensor", "achieved": tflops, "unit": "TFLOP/s",
+            "peak": peaks["bf16_tflops_sustained"], "peak_source": peaks["source"] + " (sustained bf16)",
+            "frac": tflops / peaks["bf16_tflops_sustained"],
+            "peak_nominal": NOMINAL["bf16_tflops"], "frac_of_nominal": tflops / NOMINAL["bf16_tflops"],
+            "ms": ms, "tensor_ms_at_measured_sustained": tensor_ms,
+            "sfu_exp2_count": exps, "sfu_ms_at_16_per_clk_per_sm": sfu_ms, "sfu_clock_mhz": mhz,
+            "tensor_plus_sfu_ms": tensor_ms + sfu_ms}
 
 
 def decode_grouped(a2sf, dev, G, layers, steps, reps):

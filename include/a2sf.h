@@ -379,6 +379,17 @@ int a2sf_last_device_status(void *cuda_stream);
 #define A2SF_SELFTEST_MAX_WAIT_CYCLES 2000000000ll
 int a2sf_selftest_bounded_wait(int32_t which, int64_t limit_cycles, int64_t *report, void *cuda_stream);
 
+/* Bounds-checked debug library (built with -DA2SF_DEBUG as liba2sf_debug.so; the paper has no
+ * counterpart).  In it every slot, position, tile-row and ring-stage index that addresses global
+ * or shared memory inside a kernel is range-checked; a violation is counted, the first one is
+ * recorded, and the offending access is skipped (nothing traps).  a2sf_debug_build returns 1 in
+ * that library and 0 in the release one.  a2sf_debug_violations synchronises the stream, writes
+ * to the HOST array report[4] = { violations since the last call, (kernel id << 32) | source
+ * line of the first one, its index, its bound } and clears the record; the release library
+ * always reports zeros. */
+int a2sf_debug_build(void);
+int a2sf_debug_violations(int64_t *report, void *cuda_stream);
+
 const char *a2sf_status_string(int status);
 
 #ifdef __cplusplus

@@ -7,12 +7,15 @@ library has not been built this module raises on import.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 from typing import Optional
 
 import torch
 
-_LIB_PATH = Path(__file__).resolve().parent / "liba2sf.so"
+# A2SF_LIBRARY=debug selects the bounds-checked build (liba2sf_debug.so, see build.py)
+_LIB_PATH = Path(__file__).resolve().parent / (
+    "liba2sf_debug.so" if os.environ.get("A2SF_LIBRARY", "") == "debug" else "liba2sf.so")
 
 A2SF_F32, A2SF_BF16, A2SF_F16 = 0, 1, 2
 _DTYPE_CODE = {torch.float32: A2SF_F32, torch.bfloat16: A2SF_BF16, torch.float16: A2SF_F16}
@@ -38,7 +41,8 @@ class A2SFError(RuntimeError):
 def _load():
     if not _LIB_PATH.exists():
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2407_20485_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2407_20485_b200.build` (add --debug "
+            "for the bounds-checked library) "
             "(there is no CPU fallback)")
     lib = ctypes.CDLL(str(_LIB_PATH))
     vp, i32, i64, f32, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float,
@@ -78,6 +82,8 @@ def _load():
         "a2sf_cache_import": (ctypes.c_int, [vp] * 8),
         "a2sf_kernel_launch_count": (ctypes.c_int64, []),
         "a2sf_last_device_status": (ctypes.c_int, [vp]),
+        "a2sf_debug_build": (ctypes.c_int, []),
+        "a2sf_debug_violations": (ctypes.c_int, [ctypes.POINTER(ctypes.c_int64), vp]),
         "a2sf_select": (ctypes.c_int, [ctypes.POINTER(a2sf_params), ctypes.c_int32, vp, vp, vp]),
         "a2sf_selftest_bounded_wait": (ctypes.c_int, [ctypes.c_int32, ctypes.c_int64, vp, vp]),
         "a2sf_status_string": (ctypes.c_char_p, [ctypes.c_int]),
@@ -132,6 +138,18 @@ def a2sf_kernel_launch_count() -> int:
 
 def a2sf_last_device_status(stream=None) -> int:
     return int(lib.a2sf_last_device_status(_stream(stream)))
+
+
+def a2sf_debug_build() -> bool:
+    return bool(lib.a2sf_debug_build())
+
+
+def a2sf_debug_violations(stream=None):
+    """(count, kernel id, source line, index, bound) of the bounds-checked debug library since the
+    last call; all zero in the release library."""
+    rep = (ctypes.c_int64 * 4)()
+    _check(lib.a2sf_debug_violations(rep, _stream(stream)), "a2sf_debug_violations")
+    return int(rep[0]), int(rep[1]) >> 32, int(rep[1]) & 0xffffffff, int(rep[2]), int(rep[3])
 
 
 def a2sf_select(p: a2sf_params, scores: torch.Tensor, kept_idx=None, stream=None) -> torch.Tensor:

@@ -6,12 +6,36 @@
 #include <mutex>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 
 namespace a2sf {
 
+TraceRange::TraceRange(const char *name) { nvtxRangePushA(name); }
+TraceRange::~TraceRange() { nvtxRangePop(); }
+
 static std::atomic<int64_t> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+#ifdef A2SF_DEBUG
+namespace {
+struct DebugReaders {
+    DebugReader fn[32];
+    int n;
+};
+DebugReaders &debug_readers()
+{
+    static DebugReaders r = {{}, 0};      // constructed on first use: registration runs during static initialisation
+    return r;
+}
+}  // namespace
+void register_debug_reader(DebugReader fn)
+{
+    DebugReaders &r = debug_readers();
+    if (r.n < 32) r.fn[r.n++] = fn;
+}
+#endif
 
 static inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
 static inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
@@ -125,6 +149,7 @@ static int prefill_impl(const a2sf_params *p, int32_t n, const void *q, const vo
                         void *out, float *scores, int32_t *kept_idx, float *lse_opt, void *workspace,
                         size_t workspace_bytes, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_prefill");
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
     if (n < 1 || !q || !k || !v || !out || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
@@ -187,6 +212,7 @@ int a2sf_prefill_group(const a2sf_params *p, int32_t group, int32_t n, const voi
                        float *scores, int32_t *kept_idx, float *lse_opt, void *workspace,
                        size_t workspace_bytes, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_prefill_group");
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
     if (group < 1 || group > A2SF_MAX_GROUP) return A2SF_ERR_UNSUPPORTED;
@@ -245,6 +271,7 @@ static int rescore_impl(const a2sf_params *p, int32_t n, const void *q, const vo
                         float *scores, int32_t *kept_idx, void *workspace, size_t workspace_bytes,
                         void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_rescore");
     (void)workspace; (void)workspace_bytes;
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
@@ -285,6 +312,7 @@ int a2sf_rescore_per_head(const a2sf_params *p, int32_t n, const void *q, const 
 
 int a2sf_select(const a2sf_params *p, int32_t n, const float *scores, int32_t *kept_idx, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_select");
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
     if (n < 1 || !scores || !kept_idx || !aligned(scores, 4) || !aligned(kept_idx, 4)) return A2SF_ERR_INVALID_ARG;
@@ -309,6 +337,7 @@ int a2sf_prefill_host(const a2sf_params *p, int32_t n, const void *q_host, const
                       void **dev_k, void **dev_v, float **dev_scores, int32_t **dev_kept,
                       void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_prefill_host");
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;
     if (n < 1 || !q_host || !k_host || !v_host || !out_host || !scores_host || !kept_idx_host)
@@ -486,6 +515,7 @@ int a2sf_cache_load(a2sf_cache *cache, int32_t n, const void *k, const void *v, 
                     int64_t stride_h, int64_t stride_t, const float *scores,
                     const int32_t *kept_idx, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_cache_load");
     if (!cache || n < 1 || !k || !v || !scores || !kept_idx) return A2SF_ERR_INVALID_ARG;
     int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
     if (rc != A2SF_OK) return rc;
@@ -499,6 +529,7 @@ int a2sf_cache_load(a2sf_cache *cache, int32_t n, const void *k, const void *v, 
 int a2sf_decode_step(a2sf_cache *cache, float alpha, const void *q, const void *k_new,
                      const void *v_new, void *out, int32_t *evicted_slot, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_decode_step");
     if (!cache || !q || !k_new || !v_new || !out || !evicted_slot) return A2SF_ERR_INVALID_ARG;
     if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16))
@@ -535,6 +566,7 @@ int a2sf_decode_multi(a2sf_cache *cache, float alpha, int32_t steps, const void 
                       const void *v_new, int64_t stride_b, int64_t stride_h, int64_t stride_t,
                       void *out, int32_t *evicted_opt, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_decode_multi");
     if (!cache || steps < 1 || !q || !k_new || !v_new || !out) return A2SF_ERR_INVALID_ARG;
     if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
     int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
@@ -562,6 +594,7 @@ int a2sf_prefill_streaming(a2sf_cache *cache, float alpha, int32_t n, const void
                            const void *v, int64_t stride_b, int64_t stride_h, int64_t stride_t,
                            void *out, int32_t *evicted_opt, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_prefill_streaming");
     if (!cache || n < 1 || !q || !k || !v || !out) return A2SF_ERR_INVALID_ARG;
     if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
     int rc = check_strides(&cache->p, stride_b, stride_h, stride_t);
@@ -585,6 +618,7 @@ int a2sf_ideal_similarity(a2sf_cache *cache, float alpha, int32_t n, const void 
                           void *out, float *cos_out, int32_t *evicted_opt, void *workspace,
                           size_t workspace_bytes, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_ideal_similarity");
     if (!cache || n < 1 || !q || !k || !v || !out || !cos_out) return A2SF_ERR_INVALID_ARG;
     if (n > A2SF_IDEAL_SIMILARITY_MAX_N) return A2SF_ERR_UNSUPPORTED;
     if (!(alpha >= 0.f && alpha <= 1.f)) return A2SF_ERR_INVALID_ARG;
@@ -606,6 +640,7 @@ int a2sf_ideal_similarity(a2sf_cache *cache, float alpha, int32_t n, const void 
 int a2sf_decode_step_group(a2sf_cache *cache, int32_t group, float alpha, const void *q, const void *k_new,
                            const void *v_new, void *out, int32_t *evicted_slot, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_decode_step_group");
     if (!cache || !q || !k_new || !v_new || !out || !evicted_slot) return A2SF_ERR_INVALID_ARG;
     if (group < 1 || group > A2SF_MAX_GROUP) return A2SF_ERR_UNSUPPORTED;
     if (decode_group_smem_bytes(cache->view.M, group, cache->view.d) > 220 * 1024) return A2SF_ERR_UNSUPPORTED;
@@ -622,6 +657,7 @@ int a2sf_decode_step_per_head(a2sf_cache *cache, const float *alphas, const void
                               const void *k_new, const void *v_new, void *out,
                               int32_t *evicted_slot, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_decode_step_per_head");
     if (!cache || !alphas || !q || !k_new || !v_new || !out || !evicted_slot)
         return A2SF_ERR_INVALID_ARG;
     if (!aligned(alphas, 4) || !aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) ||
@@ -650,6 +686,7 @@ int a2sf_decode_step_host(a2sf_cache *cache, float alpha, const void *q_host,
                           const void *k_new_host, const void *v_new_host, void *out_host,
                           int32_t *evicted_slot_host, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_decode_step_host");
     if (!cache || !q_host || !k_new_host || !v_new_host || !out_host || !evicted_slot_host)
         return A2SF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -693,6 +730,7 @@ static int copy_part(void *dst, const void *src, size_t bytes, cudaStream_t s)
 int a2sf_cache_export(const a2sf_cache *cache, void *k, void *v, float *scores, int32_t *pos,
                       int32_t *count, int32_t *len, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_cache_export");
     if (!cache) return A2SF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const CacheView &c = cache->view;
@@ -710,6 +748,7 @@ int a2sf_cache_import(a2sf_cache *cache, const void *k, const void *v, const flo
                       const int32_t *pos, const int32_t *count, const int32_t *len,
                       void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_cache_import");
     if (!cache) return A2SF_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const CacheView &c = cache->view;
@@ -742,6 +781,36 @@ int a2sf_selftest_bounded_wait(int32_t which, int64_t limit_cycles, int64_t *rep
     if (launch_wait_probe(word, (long long)limit_cycles, reinterpret_cast<long long *>(report),
                           static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
         return A2SF_ERR_CUDA;
+    return A2SF_OK;
+}
+
+int a2sf_debug_build(void)
+{
+#ifdef A2SF_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int a2sf_debug_violations(int64_t *report, void *cuda_stream)
+{
+    if (!report) return A2SF_ERR_INVALID_ARG;
+    report[0] = report[1] = report[2] = report[3] = 0;
+#ifdef A2SF_DEBUG
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    DebugReaders &r = debug_readers();
+    for (int i = 0; i < r.n; ++i) {
+        unsigned long long rec[4] = {0, 0, 0, 0};
+        if (r.fn[i](rec, s) != 0) return A2SF_ERR_CUDA;
+        if (rec[0] != 0 && report[0] == 0) {
+            report[1] = (int64_t)rec[1]; report[2] = (int64_t)rec[2]; report[3] = (int64_t)rec[3];
+        }
+        report[0] += (int64_t)rec[0];
+    }
+#else
+    (void)cuda_stream;
+#endif
     return A2SF_OK;
 }
 

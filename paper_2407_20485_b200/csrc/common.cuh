@@ -106,6 +106,69 @@ __device__ __forceinline__ unsigned long long warp_min_u64(unsigned long long v)
     return v;
 }
 
+// ---- bounds-checked debug build (-DA2SF_DEBUG) -------------------------------------------
+// In the debug library every slot, position, tile-row and ring-stage index that addresses
+// global or shared memory passes through A2SF_IN_RANGE before it is used.  A violation is
+// counted, the first one is recorded (kernel id, source line, index, bound) in a device word
+// that a2sf_debug_violations reads, and the access is SKIPPED: nothing traps, the context stays
+// usable.  In the release library the macro is the constant `true` and costs nothing.
+enum DebugKernelId {
+    kDbgSelect = 1, kDbgCacheLoad, kDbgDecodeStream, kDbgDecodeSplit, kDbgGroupMma, kDbgGroupSimt,
+    kDbgGroupSum, kDbgPrefillSimt1, kDbgPrefillSimt2, kDbgAttnTc, kDbgScoreTc, kDbgVToHalf,
+    kDbgIdealStats, kDbgSimilarityRow
+};
+#ifdef A2SF_DEBUG
+// one record per translation unit (no relocatable device code): {violations, kernel << 32 | line,
+// index, bound}
+static __device__ unsigned long long g_dbg_record[4];
+__device__ __forceinline__ bool dbg_in_range(long long idx, long long bound, int kernel_id, int line)
+{
+    if (idx >= 0 && idx < bound) return true;
+    if (atomicAdd(&g_dbg_record[0], 1ull) == 0ull) {
+        g_dbg_record[1] = ((unsigned long long)kernel_id << 32) | (unsigned)line;
+        g_dbg_record[2] = (unsigned long long)idx;
+        g_dbg_record[3] = (unsigned long long)bound;
+    }
+    return false;
+}
+#define A2SF_IN_RANGE(idx, bound, kernel_id) \
+    (::a2sf::dbg_in_range((long long)(idx), (long long)(bound), (kernel_id), __LINE__))
+// Host side: every translation unit with kernels registers a reader of its record.
+typedef int (*DebugReader)(unsigned long long *out4, cudaStream_t s);
+void register_debug_reader(DebugReader fn);
+#define A2SF_DEBUG_TRANSLATION_UNIT(name)                                                              \
+    namespace {                                                                                        \
+    int dbg_read_##name(unsigned long long *out4, cudaStream_t s)                                      \
+    {                                                                                                  \
+        const unsigned long long zero[4] = {0, 0, 0, 0};                                               \
+        if (cudaMemcpyFromSymbolAsync(out4, g_dbg_record, sizeof(zero), 0, cudaMemcpyDeviceToHost, s) != cudaSuccess ||  \
+            cudaStreamSynchronize(s) != cudaSuccess)                                                   \
+            return -1;                                                                                 \
+        if (out4[0] != 0 &&                                                                            \
+            (cudaMemcpyToSymbolAsync(g_dbg_record, zero, sizeof(zero), 0, cudaMemcpyHostToDevice, s) != cudaSuccess ||  \
+             cudaStreamSynchronize(s) != cudaSuccess))                                                 \
+            return -1;                                                                                 \
+        return 0;                                                                                      \
+    }                                                                                                  \
+    struct DbgRegistrar_##name {                                                                       \
+        DbgRegistrar_##name() { ::a2sf::register_debug_reader(&dbg_read_##name); }                     \
+    } dbg_registrar_##name;                                                                            \
+    }
+#else
+#define A2SF_IN_RANGE(idx, bound, kernel_id) (true)
+#define A2SF_DEBUG_TRANSLATION_UNIT(name)
+#endif
+
+// ---- tracing: an NVTX range around each entry point of the C ABI ---------------------------
+// (header-only NVTX: without a profiler attached a range costs one pointer test)
+struct TraceRange {
+    explicit TraceRange(const char *name);
+    ~TraceRange();
+    TraceRange(const TraceRange &) = delete;
+    TraceRange &operator=(const TraceRange &) = delete;
+};
+#define A2SF_TRACE(name) ::a2sf::TraceRange a2sf_trace_range_(name)
+
 // ---- host-side launch bookkeeping -------------------------------------------
 void count_launch(int n = 1);
 

@@ -14,6 +14,8 @@ namespace a2sf {
 
 namespace cg = cooperative_groups;
 
+A2SF_DEBUG_TRANSLATION_UNIT(decode_step)
+
 // sticky device-side status of the decode kernels (a bounded wait that ran out)
 static __device__ int g_decode_status = 0;
 
@@ -157,7 +159,8 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         for (int x = 0; x < kU; ++x) {
             const int row = ((bidx * kU + x) * NW + warp) * RPW + rsel;
             r[x] = make_uint4(0, 0, 0, 0);
-            if (bidx < nb && row < nloc) r[x] = ld_stream16_rw(base + (size_t)(s0 + row) * D + sub * VEC);
+            if (bidx < nb && row < nloc && A2SF_IN_RANGE(s0 + row, M, kDbgDecodeSplit))
+                r[x] = ld_stream16_rw(base + (size_t)(s0 + row) * D + sub * VEC);
         }
     };
     // batch index b: K batch b for b < nb, V batch b - nb after that
@@ -181,7 +184,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
             for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
             for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-            if (sub == 0 && row < nloc) w[row] = dot * c.scale;
+            if (sub == 0 && row < nloc && A2SF_IN_RANGE(row, per_max + 1, kDbgDecodeSplit)) w[row] = dot * c.scale;
         }
     };
     for (int b = 0; b < nb; b += 2) {
@@ -198,7 +201,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
         for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
         for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        if (lane == 0) w[nloc] = dot * c.scale;
+        if (lane == 0 && A2SF_IN_RANGE(nloc, per_max + 1, kDbgDecodeSplit)) w[nloc] = dot * c.scale;
     }
     __syncthreads();
 
@@ -280,7 +283,7 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     auto update = [&](int s, float s_before, int ps) {
         const float a = w[s] * rescale / l;
         const float sn = fmaf(alpha, s_before, a);
-        Su[s0 + s] = sn;
+        if (A2SF_IN_RANGE(s0 + s, M, kDbgDecodeSplit)) Su[s0 + s] = sn;
         if (full && ps <= newest_evictable) {
             // scores are >= 0, so their bit patterns order like the values
             const unsigned long long key =
@@ -330,7 +333,8 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
     }
     __syncthreads();
     const int target = s_target;
-    if (target >= 0) {
+    const bool target_ok = target >= 0 && A2SF_IN_RANGE(target, M, kDbgDecodeSplit);
+    if (target_ok) {
         if (tid < LPR)
             *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
                 *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
@@ -338,8 +342,8 @@ decode_step_split_kernel(CacheView c, float alpha_all, const float *__restrict__
             *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
                 *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
     }
-    if (tid == 0) {
-        if (target >= 0) {
+    if (tid == 0 && A2SF_IN_RANGE(u, c.U, kDbgDecodeSplit)) {
+        if (target_ok) {
             Su[target] = a_self;
             posu[target] = p;
         }
@@ -519,6 +523,9 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                     for (int r0 = 0; r0 < cnt; r0 += CR) {
                         if (!wait(&sh->empty[stage], phase ^ 1)) { alive = false; break; }
                         const uint32_t bytes = (uint32_t)min(CR, cnt - r0) * ROWB;
+                        if (!A2SF_IN_RANGE(stage, kStreamStages, kDbgDecodeStream) ||
+                            !A2SF_IN_RANGE(r0 + min(CR, cnt - r0) - 1, M, kDbgDecodeStream) ||
+                            !A2SF_IN_RANGE(u, c.U, kDbgDecodeStream)) { alive = false; *abort_flag = 1; break; }
                         tc::mbar_arrive_expect_tx(&sh->full[stage], bytes);
                         bulk_load(ring + stage * kChunkBytes, base + (size_t)r0 * ROWB, bytes, &sh->full[stage], policy);
                         ++issued;
@@ -547,7 +554,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             const bool got = wait(&sh->uq_full[qi], (n_unit / kUnitQueue) & 1);
             const int u = got ? sh->unit_q[qi] : -1;
             const int cnt = got ? sh->cnt_q[qi] : 0;
-            if (consumer_any(!got) || u < 0) break;        // uniform over the consumers
+            if (consumer_any(!got) || u < 0 || !A2SF_IN_RANGE(u, c.U, kDbgDecodeStream)) break;   // uniform over the consumers
             if (lane == 0) tc::mbar_arrive(&sh->uq_empty[qi]);
             const int p = c.len[u];
             const float alpha = unit_alpha(alpha_vec, u, alpha_all);
@@ -592,7 +599,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                     for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
                     for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    if (sub == 0 && row < cnt) w[row] = dot * c.scale;
+                    if (sub == 0 && row < cnt && A2SF_IN_RANGE(row, M + 1, kDbgDecodeStream)) w[row] = dot * c.scale;
                 }
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(&sh->empty[stage]);
@@ -606,7 +613,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                 for (int e = 0; e < VEC; ++e) dot = fmaf(qf[e], kf[e], dot);
 #pragma unroll
                 for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                if (lane == 0) w[cnt] = dot * c.scale;
+                if (lane == 0 && A2SF_IN_RANGE(cnt, M + 1, kDbgDecodeStream)) w[cnt] = dot * c.scale;
             }
             consumer_barrier();
 
@@ -686,7 +693,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                 else if (x_pre == 1) { s_old = s_pre[1]; ps = pos_pre[1]; }
                 else { s_old = Su[s_]; ps = posu[s_]; }
                 const float sn = fmaf(alpha, s_old, a);
-                if (alive) Su[s_] = sn;
+                if (alive && A2SF_IN_RANGE(s_, M, kDbgDecodeStream)) Su[s_] = sn;
                 if (full && ps <= newest_evictable) {
                     const unsigned long long key =
                         ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
@@ -709,7 +716,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
             consumer_barrier();
 
             const int target = sh->target;
-            if (target >= 0 && alive) {
+            if (target >= 0 && alive && A2SF_IN_RANGE(target, M, kDbgDecodeStream)) {
                 if (tid < LPR)
                     *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
                         *reinterpret_cast<const uint4 *>(k_new + uo + tid * VEC);
@@ -718,7 +725,7 @@ decode_step_stream_kernel(CacheView c, float alpha_all, const float *__restrict_
                         *reinterpret_cast<const uint4 *>(v_new + uo + (tid - LPR) * VEC);
             }
             if (tid == 0 && alive) {
-                if (target >= 0) {
+                if (target >= 0 && A2SF_IN_RANGE(target, M, kDbgDecodeStream)) {
                     Su[target] = a_self;
                     posu[target] = p;
                 }

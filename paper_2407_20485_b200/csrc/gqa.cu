@@ -13,6 +13,8 @@
 #include "common.cuh"
 
 namespace a2sf {
+
+A2SF_DEBUG_TRANSLATION_UNIT(gqa)
 namespace {
 
 constexpr int kGroupThreads = 256;
@@ -26,7 +28,7 @@ __global__ void group_sum_kernel(const float *__restrict__ per_head, float *__re
         const size_t u = idx / n, j = idx % n;
         float s = 0.f;
         for (int g = 0; g < G; ++g) s += per_head[(u * G + g) * (size_t)n + j];   // fixed order
-        out[idx] = s;
+        if (A2SF_IN_RANGE(idx, total, kDbgGroupSum)) out[idx] = s;
     }
 }
 
@@ -134,7 +136,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
         for (int x = 0; x < kUnroll; ++x) {
             const int s = s0 + x * NW * RPW + rsel;
             raw[x] = make_uint4(0u, 0u, 0u, 0u);
-            if (s <= cnt)
+            if (s <= cnt && A2SF_IN_RANGE(s, c.M + 1, kDbgGroupSimt))
                 raw[x] = *reinterpret_cast<const uint4 *>((s < cnt ? base + (size_t)s * D : fresh) + sub * VEC);
         }
     };
@@ -158,7 +160,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
             }
             const float tot = group_reduce<GMAX, LPR>(dot, sub);
             const int g = sub / LPG;
-            if (sub % LPG == 0 && g < G && s <= cnt) w[g * wstride + s] = tot * c.scale;
+            if (sub % LPG == 0 && g < G && s <= cnt && A2SF_IN_RANGE(s, wstride, kDbgGroupSimt)) w[g * wstride + s] = tot * c.scale;
         }
 #pragma unroll
         for (int x = 0; x < kUnroll; ++x) cur[x] = nxt[x];
@@ -264,7 +266,7 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
         float gain = 0.f;
         for (int g = 0; g < G; ++g) gain += w[g * wstride + s];
         const float sn = fmaf(alpha, s_old[s], gain);
-        Su[s] = sn;
+        if (A2SF_IN_RANGE(s, c.M, kDbgGroupSimt)) Su[s] = sn;
         const int ps = s_pos[s];
         if (full && ps <= newest_evictable) {
             const unsigned long long key = ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
@@ -297,15 +299,16 @@ decode_step_group_kernel(CacheView c, int G, float alpha, const T *__restrict__ 
     __syncthreads();
     const int target = s_target;
     if (target >= 0) {
-        if (tid < LPR)
+        if (!A2SF_IN_RANGE(target, c.M, kDbgGroupSimt)) {
+        } else if (tid < LPR)
             *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * VEC) =
                 *reinterpret_cast<const uint4 *>(knu + tid * VEC);
         else if (tid < 2 * LPR)
             *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * VEC) =
                 *reinterpret_cast<const uint4 *>(vnu + (tid - LPR) * VEC);
     }
-    if (tid == 0) {
-        if (target >= 0) {
+    if (tid == 0 && A2SF_IN_RANGE(u, c.U, kDbgGroupMma)) {
+        if (target >= 0 && A2SF_IN_RANGE(target, c.M, kDbgGroupMma)) {
             Su[target] = s_new;
             posu[target] = p;
         }
@@ -437,7 +440,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
 #pragma unroll
             for (int j = 0; j < KL; ++j) {
                 buf[h][j] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile < ntile && s <= cnt)
+                if (tile < ntile && s <= cnt && A2SF_IN_RANGE(s, c.M + 1, kDbgGroupMma))
                     buf[h][j] = *reinterpret_cast<const uint4 *>(row_ptr(s, Ku, knu) + 32 * j + 8 * cq);
             }
         }
@@ -495,7 +498,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
 #pragma unroll
             for (int i = 0; i < VL; ++i) {
                 buf[x][i] = make_uint4(0u, 0u, 0u, 0u);
-                if (tile < ntile && s <= cnt)
+                if (tile < ntile && s <= cnt && A2SF_IN_RANGE(s, c.M + 1, kDbgGroupMma))
                     buf[x][i] = *reinterpret_cast<const uint4 *>(row_ptr(s, Vu, vnu) + E * r + 8 * i);
             }
         }
@@ -517,7 +520,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
 #pragma unroll 4
         for (int s = tid >> 3; s < nrow; s += kGroupThreads / 8) {
             const float e = g < G ? expf(w[s * kMmaCols + g] - m) : 0.f;   // unused columns 0
-            w[s * kMmaCols + g] = e;
+            if (A2SF_IN_RANGE(s, c.M + 1, kDbgGroupMma)) w[s * kMmaCols + g] = e;
             l += e;
         }
         l += __shfl_xor_sync(0xffffffffu, l, 8);
@@ -604,7 +607,7 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
         float gain = 0.f;
         for (int g = 0; g < G; ++g) gain += w[(size_t)s * kMmaCols + g] * s_inv[g];
         const float sn = fmaf(alpha, s_old[s], gain);
-        Su[s] = sn;
+        if (A2SF_IN_RANGE(s, c.M, kDbgGroupSimt)) Su[s] = sn;
         const int ps = s_pos[s];
         if (full && ps <= newest_evictable) {
             const unsigned long long key = ((unsigned long long)__float_as_uint(sn) << 32) | (unsigned)ps;
@@ -638,15 +641,16 @@ decode_step_group_mma_kernel(CacheView c, int G, float alpha, const T *__restric
     const int target = s_target;
     if (target >= 0) {
         constexpr int LPR = D / 8;
-        if (tid < LPR)
+        if (!A2SF_IN_RANGE(target, c.M, kDbgGroupMma)) {
+        } else if (tid < LPR)
             *reinterpret_cast<uint4 *>(Ku + (size_t)target * D + tid * 8) =
                 *reinterpret_cast<const uint4 *>(knu + tid * 8);
         else if (tid < 2 * LPR)
             *reinterpret_cast<uint4 *>(Vu + (size_t)target * D + (tid - LPR) * 8) =
                 *reinterpret_cast<const uint4 *>(vnu + (tid - LPR) * 8);
     }
-    if (tid == 0) {
-        if (target >= 0) {
+    if (tid == 0 && A2SF_IN_RANGE(u, c.U, kDbgGroupMma)) {
+        if (target >= 0 && A2SF_IN_RANGE(target, c.M, kDbgGroupMma)) {
             Su[target] = s_new;
             posu[target] = p;
         }

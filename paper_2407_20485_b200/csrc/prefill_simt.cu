@@ -10,6 +10,8 @@
 
 namespace a2sf {
 
+A2SF_DEBUG_TRANSLATION_UNIT(prefill_simt)
+
 namespace {
 
 constexpr int kRows = 32;       // query rows (pass 1) / keys (pass 2) per CTA, 4 threads each
@@ -132,7 +134,7 @@ __global__ void __launch_bounds__(kThreads) prefill_pass1_simt(PrefillArgs a)
         }
         m = m_new;
     }
-    if (valid) {
+    if (valid && A2SF_IN_RANGE(i, a.n, kDbgPrefillSimt1)) {
         const float inv = 1.f / l;
         T *orow = O + (int64_t)i * a.st.t;
 #pragma unroll
@@ -193,7 +195,7 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
                 const int age = a.n - 1 - i;
                 cv = lse[i] * kLog2e + (age == 0 ? 0.f : (float)age * neg_log2_alpha);
             }
-            cs[threadIdx.x] = cv;
+            if (A2SF_IN_RANGE(threadIdx.x, kTile, kDbgPrefillSimt2)) cs[threadIdx.x] = cv;
         }
         __syncthreads();
 #pragma unroll 8
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(kThreads) prefill_pass2_simt(PrefillArgs a)
             acc += (i0 + ii >= j) ? pw : 0.f;         // causal: rows i >= j only
         }
     }
-    if (valid && tq == 0) a.scores[(int64_t)u * a.n + j] = acc;
+    if (valid && tq == 0 && A2SF_IN_RANGE(j, a.n, kDbgPrefillSimt2)) a.scores[(int64_t)u * a.n + j] = acc;
 }
 
 template <typename T, int D>

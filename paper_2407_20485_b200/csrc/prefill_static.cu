@@ -54,6 +54,7 @@ extern "C" int a2sf_prefill_static_scratch(const a2sf_params *p, int32_t n, cons
                                            int64_t stride_h, int64_t stride_t, void *out,
                                            float *scores, int32_t *kept_idx, void *cuda_stream)
 {
+    A2SF_TRACE("a2sf_prefill_static_scratch");
     // the same checks, in the same order, as a2sf_prefill
     int rc = check_params(p);
     if (rc != A2SF_OK) return rc;

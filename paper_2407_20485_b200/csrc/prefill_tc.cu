@@ -19,6 +19,8 @@
 
 namespace a2sf {
 
+A2SF_DEBUG_TRANSLATION_UNIT(prefill_tc)
+
 // sticky device-side status: set when a bounded wait runs out
 static __device__ int g_tc_status = 0;
 
@@ -247,8 +249,9 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             issued = max(issued, it + 1);
-            *reinterpret_cast<float4 *>(&sh->cbuf[it % kScoreCRing][lane * 4]) =
-                make_float4(c4[0], c4[1], c4[2], c4[3]);
+            if (A2SF_IN_RANGE(lane * 4 + 3, kBlk, kDbgScoreTc))
+                *reinterpret_cast<float4 *>(&sh->cbuf[it % kScoreCRing][lane * 4]) =
+                    make_float4(c4[0], c4[1], c4[2], c4[3]);
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->c_ready[it % kScoreCRing]);
         }
@@ -318,7 +321,9 @@ score_pass_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant_
         }
         if (hsel == 1) sh->part[key_lane] = sum;
         named_barrier(1, kScoreEpiThreads);
-        if (hsel == 0 && j < a.n && !*abort_flag) a.scores[(size_t)u * a.n + j] = sum + sh->part[key_lane];
+        if (hsel == 0 && j < a.n && !*abort_flag && A2SF_IN_RANGE(key_lane, kBlk, kDbgScoreTc) &&
+            A2SF_IN_RANGE((size_t)u * a.n + j, (size_t)gridDim.x / ntile_total * a.n, kDbgScoreTc))
+            a.scores[(size_t)u * a.n + j] = sum + sh->part[key_lane];
     }
 
     tc_fence_before_sync();
@@ -511,6 +516,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
             int k_issued = 1, v_issued = 1;
             for (int t = 1; t < nt; ++t) {
                 const int ks = t % kKStages, vs = t % kVStages;
+                if (!A2SF_IN_RANGE(t * kBlk, a.n, kDbgAttnTc)) break;      // a tile past the prompt is never requested
                 if (!wait(&sh->k_empty[ks], ((t / kKStages) & 1) ^ 1)) break;
                 mbar_arrive_expect_tx(&sh->k_full[ks], kTileBytes);
                 tma_load_4d(Ks + ks * kTileBytes, tmap_k, &sh->k_full[ks], 0, t * kBlk, hk, b);
@@ -738,7 +744,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
                 uint32_t o[32];
                 tmem_ld32(to + c * 32, o);
                 tmem_wait_ld();
-                if (i < a.n) {
+                if (i < a.n && A2SF_IN_RANGE(half * 64 + c * 32 + 31, kD, kDbgAttnTc)) {
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint32_t w[4];
@@ -750,7 +756,7 @@ __device__ __forceinline__ void attn_body(const CUtensorMap *tmap_q, const CUten
                     }
                 }
             }
-            if (half == 0 && i < a.n)
+            if (half == 0 && i < a.n && A2SF_IN_RANGE(u, gridDim.x / npairs, kDbgAttnTc))
                 a.lse[(size_t)u * a.n + i] = (m_used[X] + log2f(lsum)) * 0.6931471805599453f;
         };
         finish(std::integral_constant<int, 0>{}, ntA, rbA);
@@ -815,7 +821,7 @@ __global__ void v_to_half_kernel(const __nv_bfloat16 *__restrict__ v, Strides st
             bad |= !(fabsf(f[2 * e]) <= 65504.f) | !(fabsf(f[2 * e + 1]) <= 65504.f);   // also NaN
             oh[e] = __floats2half2_rn(f[2 * e], f[2 * e + 1]);
         }
-        *reinterpret_cast<uint4 *>(dst + idx * 8) = o;
+        if (A2SF_IN_RANGE(idx, chunks, kDbgVToHalf)) *reinterpret_cast<uint4 *>(dst + idx * 8) = o;
     }
     if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1);
 }

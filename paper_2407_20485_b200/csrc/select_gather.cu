@@ -6,6 +6,8 @@
 
 namespace a2sf {
 
+A2SF_DEBUG_TRANSLATION_UNIT(select_gather)
+
 namespace {
 
 constexpr int kSelThreads = 1024;
@@ -56,7 +58,8 @@ select_kernel(const float *__restrict__ scores, int32_t *__restrict__ kept, int 
     const int tid = threadIdx.x;
 
     if (n <= M) {
-        for (int j = tid; j < n; j += kSelThreads) out[j] = j;
+        for (int j = tid; j < n; j += kSelThreads)
+            if (A2SF_IN_RANGE(j, min(n, M), kDbgSelect)) out[j] = j;
         return;
     }
     const int ncand = n - R;
@@ -70,7 +73,7 @@ select_kernel(const float *__restrict__ scores, int32_t *__restrict__ kept, int 
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
         for (int j = tid; j < ncand; j += kSelThreads) {
-            const unsigned bits = S[j];
+            const unsigned bits = A2SF_IN_RANGE(j, n, kDbgSelect) ? S[j] : 0u;
             if ((bits & mask) == prefix) atomicAdd(&hist[(bits >> shift) & 255u], 1);
         }
         __syncthreads();
@@ -97,7 +100,7 @@ select_kernel(const float *__restrict__ scores, int32_t *__restrict__ kept, int 
         const int j = j0 + tid;
         unsigned bits = 0;
         bool cand = false;
-        if (j < n) { bits = S[j]; cand = j < ncand; }
+        if (j < n && A2SF_IN_RANGE(j, n, kDbgSelect)) { bits = S[j]; cand = j < ncand; }
         const int is_eq = (cand && bits == thr) ? 1 : 0;
         int eq_total;
         const int eq_before = eq_base + block_excl_scan(is_eq, warp_tot, eq_total);
@@ -105,7 +108,7 @@ select_kernel(const float *__restrict__ scores, int32_t *__restrict__ kept, int 
         if (j < n) keep = !cand || bits > thr || (is_eq && eq_before >= eq_drop);
         int keep_total;
         const int kpos = kept_base + block_excl_scan(keep ? 1 : 0, warp_tot, keep_total);
-        if (keep && kpos < M) out[kpos] = j;
+        if (keep && kpos < M && A2SF_IN_RANGE(kpos, min(n, M), kDbgSelect)) out[kpos] = j;
         kept_base += keep_total;
         eq_base += eq_total;
     }
@@ -122,12 +125,13 @@ __global__ void cache_load_kernel(CacheView c, int H, int n, const char *__restr
     const int slot = blockIdx.y * warps_per_block + (threadIdx.x >> 5);
     const int u = blockIdx.x;
     const int lane = threadIdx.x & 31;
-    if (slot >= c.M) return;
+    if (slot >= c.M || !A2SF_IN_RANGE(u, c.U, kDbgCacheLoad)) return;
     const int m = min(n, c.M);
     char *Kc = static_cast<char *>(c.K) + ((size_t)u * c.M + slot) * ROW_BYTES;
     char *Vc = static_cast<char *>(c.V) + ((size_t)u * c.M + slot) * ROW_BYTES;
     if (slot < m) {
         int j = kept[(size_t)u * m + slot];
+        (void)A2SF_IN_RANGE(j, n, kDbgCacheLoad);      // debug build: a kept index outside the prompt is reported
         j = min(max(j, 0), n - 1);        // a corrupt index must not leave the tensor
         const int b = u / H, h = u % H;
         const int64_t off = b * st_bytes.b + h * st_bytes.h + (int64_t)j * st_bytes.t;

@@ -17,6 +17,8 @@
 #include "common.cuh"
 
 namespace a2sf {
+
+A2SF_DEBUG_TRANSLATION_UNIT(similarity)
 namespace {
 
 constexpr int kSimThreads = 256;
@@ -117,7 +119,7 @@ ideal_stats_kernel(const T *__restrict__ q, const T *__restrict__ k, Strides st,
     float mx = -INFINITY;
     for (int j = threadIdx.x; j <= i; j += kSimThreads) {
         const float s = row_dot<T, D>(qs, k + base + (size_t)j * st.t) * scale;
-        logit[j] = s;
+        if (A2SF_IN_RANGE(j, n, kDbgIdealStats)) logit[j] = s;
         mx = fmaxf(mx, s);
     }
     const float m = block_max(mx, red);
@@ -160,6 +162,7 @@ ideal_stats_kernel(const T *__restrict__ q, const T *__restrict__ k, Strides st,
     n2 = block_sum(n2, red);
     if (threadIdx.x == 0) {
         const size_t o = (size_t)u * n + i;
+        if (!A2SF_IN_RANGE(i, n, kDbgIdealStats)) return;
         out.thr[o] = keep < i + 1 ? from_ordered_bits((uint32_t)(thr_key >> 32)) : -INFINITY;
         out.thr_pos[o] = keep < i + 1 ? (int32_t)(0xffffffffu - (uint32_t)(thr_key & 0xffffffffu)) : INT_MAX;
         out.m[o] = m;
@@ -187,7 +190,7 @@ similarity_row_kernel(CacheView c, const T *__restrict__ q, const T *__restrict_
     float mx = -INFINITY;
     for (int s = threadIdx.x; s <= cnt; s += kSimThreads) {
         const float v = row_dot<T, D>(qs, s < cnt ? Ku + (size_t)s * D : k_new + uo) * c.scale;
-        w[s] = v;
+        if (A2SF_IN_RANGE(s, c.M + 1, kDbgSimilarityRow)) w[s] = v;
         mx = fmaxf(mx, v);
     }
     const float m_meth = block_max(mx, red);
@@ -204,7 +207,7 @@ similarity_row_kernel(CacheView c, const T *__restrict__ q, const T *__restrict_
     }
     a2 = block_sum(a2, red);
     dot = block_sum(dot, red);
-    if (threadIdx.x == 0) cos_out[o] = dot / sqrtf(a2 * ideal.n2[o]);
+    if (threadIdx.x == 0 && A2SF_IN_RANGE(i, n, kDbgSimilarityRow)) cos_out[o] = dot / sqrtf(a2 * ideal.n2[o]);
 }
 
 template <typename T, int D>
