@@ -411,6 +411,9 @@ def run_ours(args):
         # grouped query heads (not part of the headline): the same policy on 8 K/V heads per row
         result["decode_grouped"] = [decode_grouped(a2sf, dev, G, 8, args.rotation_steps, args.rotation_reps)
                                     for G in (4, 8)]
+        # the same step at five times the batch: 1280 units, 345 MB per launch, several rounds of CTAs
+        result["decode_grouped"] += [decode_grouped(a2sf, dev, G, 1, args.rotation_steps, args.rotation_reps, B=160)
+                                     for G in (4, 8)]
     if rank == 0:
         print(json.dumps(result))
     a2dist.finalize()
@@ -439,12 +442,12 @@ def prefill_roofline(w, U, tflops, ms, peaks, sm_mhz):
             "tensor_plus_sfu_ms": tensor_ms + sfu_ms}
 
 
-def decode_grouped(a2sf, dev, G, layers, steps, reps):
+def decode_grouped(a2sf, dev, G, layers, steps, reps, B=None):
     """Grouped-query decode step (G query heads per K/V head, one pruned cache per K/V head) on the
     headline workload's policy with 8 K/V heads per batch row: 256 units x 512 slots, 69 MB per
     launch.  Timed like `decode_layer_rotation`: one layer (fits in L2) and `layers` caches stepped
     round-robin (larger than L2), `steps` x layers launches replayed from a CUDA graph."""
-    w = wl.WORKLOADS["llama2_13b"].scaled(H=8, n=1024)
+    w = wl.WORKLOADS["llama2_13b"].scaled(H=8, n=1024, **({"B": B} if B else {}))
     wq = w.scaled(H=w.H * G)
     q = wl.make_prompt(wq, dev)[0]
     _, k, v = wl.make_prompt(w, dev)

@@ -461,6 +461,9 @@ def test_streamed_prompt_against_the_oracle(name, kw):
     ("opt_6p7b", dict(B=9, H=8, n=140, budget=70, recent=0, steps=16), 8),
     ("tiny_fp32", dict(B=16, H=5, n=100, budget=40, recent=20, steps=12), 2),
     ("llama2_13b", dict(B=4, H=16, n=130, budget=300, recent=100, steps=12, d=64), 5),   # appends only, d = 64
+    # more units than CTAs that run at once: every persistent CTA walks several units
+    ("llama2_7b", dict(B=41, H=8, n=100, budget=48, recent=24, steps=10), 4),
+    ("opt_6p7b", dict(B=20, H=37, n=70, budget=80, recent=0, steps=14, d=64), 3),
     # 16-bit storage runs the group's products on the tensor cores, fp32 storage on CUDA cores
     # (instantiated for group bounds 2, 4 and 8): a ragged last tile of slots, d = 64, a group of one
     ("opt_6p7b", dict(B=1, H=3, n=200, budget=77, recent=30, steps=30, d=64), 6),
