@@ -25,7 +25,8 @@ SWEEP = ("tiny_fp32_full or shrunken_configs or edge_cases or random_shapes or g
 def test_small_shape_sweep_under_the_bounds_checked_library_with_guard_words():
     from paper_2407_20485_b200 import build
 
-    assert build.DEBUG_LIB_PATH.exists(), "build it with `python -m paper_2407_20485_b200.build --debug`"
+    build.build(debug=True)          # incremental: a no-op when liba2sf_debug.so is up to date
+    assert build.DEBUG_LIB_PATH.exists()
     env = dict(os.environ, A2SF_LIBRARY="debug", A2SF_GUARDS="1")
     cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
            "tests/test_parity_gpu.py", "-k", SWEEP]
@@ -79,6 +80,9 @@ torch.cuda.synchronize()
 assert int(st["pos"][0, 1, 5]) == w.n - 1            # clamped into the prompt, as in the release library
 print("positive control ok")
 '''
+    from paper_2407_20485_b200 import build
+
+    build.build(debug=True)
     env = dict(os.environ, A2SF_LIBRARY="debug")
     r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0 and "positive control ok" in r.stdout, r.stdout[-2000:] + r.stderr[-3000:]
